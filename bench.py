@@ -1,0 +1,430 @@
+#!/usr/bin/env python
+"""Benchmark of the fused attention-weight kernel (and, beside it, the dedicated row-Softmax kernel).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one launch of ``attnw_fused`` over the whole headline workload (fused, B=4, H=32,
+N=4096, d=128, bf16 -> bf16 P): matmul, scaling, statistics pass, normalise pass and the store of P.
+``value`` is attention-weight elements per second with inputs resident in HBM; ``e2e`` is the same
+metric through the host-buffer C-ABI call (host->device and device->host copies inside the timed
+region).  With N > 1 (torchrun) every rank runs the full workload on its own seeded inputs (heads are
+independent, no collective on the data path): weak scaling, time = max over ranks.
+
+``--impl reference`` times the CPU oracle on the host cores on a bounded sample of the same workload.
+Prints exactly one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "attention-weight elements/sec"
+UNIT = "elements/s"
+HEADLINE = "c3"
+# Fallback peaks (an earlier measurement on this machine) used only when MEASURED_PEAKS.json is absent.
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
+# summarised under profiles/; None until a capture exists for that kernel.
+NCU_TRAFFIC_BYTES = {"c3": None, "c4": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    except Exception:
+        return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS,
+                "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons of one GPU while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, device_index: int, period_s: float = 0.002):
+        super().__init__(daemon=True)
+        self.period = period_s
+        self.samples: list[int] = []
+        self.reason_bits = 0
+        self.sm_max = None
+        self.halt = threading.Event()
+        self.handle = None
+        self.nvml = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            handle = None
+            try:
+                uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+                if not uuid.startswith("GPU-"):
+                    uuid = "GPU-" + uuid
+                handle = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                handle = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.handle = handle
+            self.nvml = pynvml
+            self.sm_max = int(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.handle = None
+
+    def _reasons(self) -> int:
+        n = self.nvml
+        for name in ("nvmlDeviceGetCurrentClocksEventReasons", "nvmlDeviceGetCurrentClocksThrottleReasons"):
+            fn = getattr(n, name, None)
+            if fn is not None:
+                try:
+                    return int(fn(self.handle))
+                except Exception:
+                    continue
+        return 0
+
+    def run(self):
+        if self.handle is None:
+            return
+        n = self.nvml
+        while not self.halt.is_set():
+            try:
+                self.samples.append(int(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM)))
+                self.reason_bits |= self._reasons()
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def summary(self) -> dict:
+        if self.handle is None or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": [], "samples": 0,
+                    "note": "NVML unavailable" if self.handle is None else "no samples"}
+        reasons = [name for bit, name in self.REASONS.items() if self.reason_bits & bit]
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.sm_max, "reasons": reasons,
+                "samples": len(self.samples)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle legs (the only places this file touches oracle/)
+# ------------------------------------------------------------------------------------------
+
+def oracle_sample_rate(w, target_seconds: float, seed_offset: int = 0):
+    """Times the oracle, as it stands, on complete rows of the workload; returns (elements/s, info)."""
+    import oracle
+    from paper_2407_13885_b200 import inputs
+    cores = oracle.host_cores()
+    heads = min(2, w.B * w.H)
+    q, k = inputs.make_qk(w, 0, heads)
+    q = q.reshape(1, heads, w.N, w.d)
+    k = k.reshape(1, heads, w.N, w.d)
+    rng = np.random.default_rng(1234 + seed_offset)
+    probe = max(cores * 8, 64)
+    ids = rng.integers(0, heads * w.N, size=probe)
+    t0 = time.perf_counter()
+    oracle.attnw_rows(q, k, w.scale, ids)
+    dt = time.perf_counter() - t0
+    per_row = dt / probe
+    n_rows = int(min(max(probe, target_seconds / max(per_row, 1e-9)), 1 << 22))
+    ids = rng.integers(0, heads * w.N, size=n_rows)
+    t0 = time.perf_counter()
+    oracle.attnw_rows(q, k, w.scale, ids)
+    dt = time.perf_counter() - t0
+    value = n_rows * w.N / dt
+    info = {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n_rows} complete rows (N={w.N}, d={w.d}) drawn from {heads} heads of {w.name}, "
+                      f"{dt:.2f} s wall, fp64, threaded over rows"}
+    return value, info, dt, n_rows
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return 0
+    from paper_2407_13885_b200 import inputs
+    w = inputs.WORKLOADS[args.workload]
+    # seconds of CPU work per step, bounded so that the whole run ends within a few minutes
+    per_step = max(0.2, min(4.0, 150.0 / max(args.steps + args.warmup, 1)))
+    for i in range(args.warmup):
+        oracle_sample_rate(w, 0.5, seed_offset=i)
+    total_t, total_rows, info = 0.0, 0, None
+    for i in range(args.steps):
+        _, info, dt, n_rows = oracle_sample_rate(w, per_step, seed_offset=100 + i)
+        total_t += dt
+        total_rows += n_rows
+    value = total_rows * w.N / total_t
+    info["value"] = value
+    info["sample"] = (f"each step = about {per_step:.0f} s of oracle work on complete rows of {w.name} "
+                      f"({total_rows} rows over {args.steps} steps)")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / max(args.steps, 1),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_config(w, 1),
+            "cpu_baseline": info,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(w, world):
+    cfg = {"workload": f"{w.name}: fused attention weights B={w.B} H={w.H} N={w.N} d={w.d}, Q,K bf16 N(0,{w.sigma:g}^2), "
+                       f"scale={w.scale:.9g}, P {w.p_dtype}",
+           "B": w.B, "H": w.H, "N": w.N, "d": w.d, "p_dtype": w.p_dtype,
+           "parallelism": f"{world} x independent replicas of the workload (heads are independent; no collective)",
+           "l2": "no flush: each launch streams 4.56 GB (Q+K 268 MB, P 4.29 GB), far beyond the 126 MB L2"}
+    return cfg
+
+
+# ------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------
+
+def time_launches(fn, steps, warmup, stream_sync):
+    """CUDA events on the current stream around `steps` back-to-back calls; returns total ms."""
+    import torch
+    for _ in range(warmup):
+        fn()
+    stream_sync()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(steps):
+        fn()
+    stop.record()
+    stop.synchronize()
+    return start.elapsed_time(stop)
+
+
+def secondary_config(binding, inputs, name, peaks, steps=20, warmup=3):
+    """Short kernel-only measurement of one of the other configurations (reported, not the headline)."""
+    import torch
+    w = inputs.WORKLOADS[name]
+    if w.kind == "rows":
+        S = torch.empty((w.rows, w.cols), dtype=torch.float32, device="cuda")
+        blk = 4096
+        for r0 in range(0, w.rows, blk):
+            S[r0:r0 + blk].copy_(torch.from_numpy(inputs.make_scores(w, r0, r0 + blk)))
+        P = torch.empty((w.rows, w.cols), dtype=torch.bfloat16, device="cuda")
+        fn = lambda: binding.softmax_rows(S, P=P)  # noqa: E731
+    else:
+        q, k = inputs.make_qk(w)
+        Q = torch.from_numpy(q.view(np.int16)).view(torch.bfloat16).reshape(w.B, w.H, w.N, w.d).cuda()
+        K = torch.from_numpy(k.view(np.int16)).view(torch.bfloat16).reshape(w.B, w.H, w.N, w.d).cuda()
+        P = torch.empty((w.B, w.H, w.N, w.N), dtype=torch.bfloat16 if w.p_dtype == "bf16" else torch.float32,
+                        device="cuda")
+        fn = lambda: binding.attnw_fused(Q, K, w.scale, P=P)  # noqa: E731
+    ms = time_launches(fn, steps, warmup, torch.cuda.synchronize) / steps
+    bytes_alg = w.in_bytes + w.p_bytes
+    t_hbm = bytes_alg / (peaks["hbm_gbs"] * 1e9)
+    t_flop = w.flops / (peaks["bf16_tflops"] * 1e12)
+    return {"elements_per_s": w.elements / (ms * 1e-3), "ms": ms, "achieved_gbs": bytes_alg / (ms * 1e-3) / 1e9,
+            "roofline_frac": max(t_hbm, t_flop) / (ms * 1e-3), "bound": "hbm" if t_hbm >= t_flop else "tensor",
+            "steps": steps}
+
+
+def run_profile_case(args):
+    """A reduced case of one kernel for profiler captures (`--profile fused|rows`): the same kernel and
+    tile configuration as the headline launch on inputs that still exceed the L2 but hold well under a
+    GB on the device.  Prints one JSON line marked as a profile run; never a benchmark value."""
+    import torch
+    from paper_2407_13885_b200 import binding, inputs
+    torch.cuda.set_device(0)
+    if args.profile == "fused":
+        base = inputs.WORKLOADS[args.workload]
+        heads = max(1, min(base.B * base.H, (512 << 20) // (base.N * base.N * 2)))
+        w = inputs.Workload(base.name + "-reduced", "fused", B=1, H=heads, N=base.N, d=base.d, sigma=base.sigma,
+                            scale=base.scale, p_dtype=base.p_dtype, cfg_id=base.cfg_id)
+        q, k = inputs.make_qk(w)
+        Q = torch.from_numpy(q.view(np.int16)).view(torch.bfloat16).reshape(1, heads, w.N, w.d).cuda()
+        K = torch.from_numpy(k.view(np.int16)).view(torch.bfloat16).reshape(1, heads, w.N, w.d).cuda()
+        P = torch.empty((1, heads, w.N, w.N), dtype=torch.bfloat16, device="cuda")
+        fn = lambda: binding.attnw_fused(Q, K, w.scale, P=P)  # noqa: E731
+        desc = f"fused B=1 H={heads} N={w.N} d={w.d} (P {w.p_bytes >> 20} MiB)"
+    else:
+        base = inputs.WORKLOADS["c4"]
+        rows = 8192
+        S = torch.from_numpy(inputs.make_scores(base, 0, rows)).cuda()
+        P = torch.empty((rows, base.cols), dtype=torch.bfloat16, device="cuda")
+        w = inputs.Workload("c4-reduced", "rows", rows=rows, cols=base.cols, sigma=base.sigma, cfg_id=4)
+        fn = lambda: binding.softmax_rows(S, P=P)  # noqa: E731
+        desc = f"softmax_rows rows={rows} cols={base.cols} (S {w.in_bytes >> 20} MiB, P {w.p_bytes >> 20} MiB)"
+    ms = time_launches(fn, args.steps, max(args.warmup, 1), torch.cuda.synchronize) / args.steps
+    print(json.dumps({"profile_run": True, "case": desc, "ms_per_launch": ms,
+                      "algorithmic_bytes_per_launch": w.in_bytes + w.p_bytes,
+                      "achieved_gbs": (w.in_bytes + w.p_bytes) / (ms * 1e-3) / 1e9, "steps": args.steps}))
+    return 0
+
+
+def run_ours(args):
+    import torch
+    from paper_2407_13885_b200 import binding, inputs  # raises if libattnw.so is missing: no fallback
+
+    rank, world, local = dist_env()
+    if world != args.gpus:
+        if world == 1 and args.gpus > 1:
+            raise SystemExit("--gpus N > 1 must be launched with torch.distributed.run (one rank per GPU)")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    w = inputs.WORKLOADS[args.workload]
+    peaks = load_peaks()
+
+    # seeded inputs: every rank draws its own replica of the workload (weak scaling)
+    q, k = inputs.make_qk(w, seed=inputs.SEED + rank)
+    shape = (w.B, w.H, w.N, w.d)
+    Qh = torch.from_numpy(q.view(np.int16)).view(torch.bfloat16).reshape(shape).pin_memory()
+    Kh = torch.from_numpy(k.view(np.int16)).view(torch.bfloat16).reshape(shape).pin_memory()
+    Q, K = Qh.cuda(), Kh.cuda()
+    p_dtype = torch.bfloat16 if w.p_dtype == "bf16" else torch.float32
+    P = torch.empty((w.B, w.H, w.N, w.N), dtype=p_dtype, device="cuda")
+
+    def step():
+        binding.attnw_fused(Q, K, w.scale, P=P)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    binding.launch_count(reset=True)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(args.steps):
+        step()
+    stop.record()
+    torch.cuda.synchronize()
+    barrier()
+    launches = binding.launch_count()
+    sampler.halt.set()
+    sampler.join()
+    elapsed_ms = start.elapsed_time(stop)
+    status = binding.query_status()
+    if status != 0:
+        raise SystemExit(f"device status word {status:#x}: a bounded wait gave up; timing is invalid")
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+        lt = torch.tensor([launches], dtype=torch.int64, device="cuda")
+        dist.all_reduce(lt, op=dist.ReduceOp.SUM)
+        launches = int(lt.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * w.elements / (ms_per_step * 1e-3)
+
+    # ---- end to end through the host-buffer C-ABI call ----
+    e2e = None
+    if not args.no_e2e:
+        Ph = torch.empty((w.B, w.H, w.N, w.N), dtype=p_dtype).pin_memory()
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        binding.host_attnw_fused(Qh, Kh, w.scale, Ph)  # warm-up: allocates the staging buffers
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            binding.host_attnw_fused(Qh, Kh, w.scale, Ph)  # returns when P is complete in host memory
+        dt = time.perf_counter() - t0
+        barrier()
+        if world > 1:
+            import torch.distributed as dist
+            t = torch.tensor([dt], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        e2e = {"value": world * w.elements * e2e_steps / dt, "unit": UNIT,
+               "h2d_bytes_per_step": w.in_bytes, "d2h_bytes_per_step": w.p_bytes,
+               "steps": e2e_steps, "ms_per_step": 1e3 * dt / e2e_steps,
+               "note": "attnw_fused_host: pinned host Q,K -> device, kernel, P -> pinned host, pipelined over "
+                       "groups of heads on two streams; wall clock around the blocking call"}
+        binding.host_release()
+        del Ph
+
+    if rank != 0:
+        return 0
+
+    bytes_alg = w.in_bytes + w.p_bytes
+    kernel_s = ms_per_step * 1e-3
+    achieved = bytes_alg / kernel_s / 1e9
+    t_hbm = bytes_alg / (peaks["hbm_gbs"] * 1e9)
+    t_flop = w.flops / (peaks["bf16_tflops"] * 1e12)
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                "peak_source": f"of {peaks['source']}",
+                "algorithmic_bytes_per_launch": bytes_alg,
+                "roofline_time_us": 1e6 * max(t_hbm, t_flop), "kernel_time_us": 1e6 * kernel_s,
+                "time_frac_of_roofline": max(t_hbm, t_flop) / kernel_s,
+                "tensor_time_us_at_burst_peak": 1e6 * t_flop,
+                "kernel": "attnw_fused_kernel<128, bf16>"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_config(w, world), "clocks": sampler.summary(), "e2e": e2e,
+            "gpu_launches": launches, "roofline": roofline}
+
+    if not args.no_cpu_baseline:
+        _, info, _, _ = oracle_sample_rate(w, args.cpu_seconds)
+        line["cpu_baseline"] = info
+    if not args.no_secondary and world == 1:
+        del P, Q, K
+        torch.cuda.empty_cache()
+        other = {}
+        for name in ("c4", "c5", "c2"):
+            other[name] = secondary_config(binding, inputs, name, peaks)
+            torch.cuda.empty_cache()
+        line["other_configs"] = other
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default=HEADLINE, choices=["c2", "c3", "c5"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true")
+    ap.add_argument("--profile", choices=["fused", "rows"], default=None,
+                    help="run a reduced case of one kernel for an ncu capture instead of the benchmark")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    if args.profile:
+        return run_profile_case(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,110 @@
+/*
+ * attnw - attention weights P = Softmax(scale * Q K^T) on NVIDIA B200 (sm_100a).
+ *
+ * C ABI of libattnw.so.  Two operations, each a hand-written CUDA kernel:
+ *
+ *   attnw_fused*   matmul + scaling + Softmax in one kernel; scores never reach HBM
+ *                  (the fused kernel of Section VII of "Attention in SRAM on Tenstorrent
+ *                  Grayskull"; the product is Attention's softmax(QK^T/sqrt(d_k)) of Section IV).
+ *   softmax_rows*  row-wise Softmax of precomputed scores (the dedicated kernel of
+ *                  Section VI-B; definition in Section VI, max subtraction of Eq. 1).
+ *
+ * Conventions shared by the device entry points
+ *   - Every data pointer is a DEVICE pointer owned by the caller; the library neither
+ *     allocates nor frees device memory in these calls.  Tensors are row-major and contiguous.
+ *   - `stream` is a cudaStream_t (NULL = the legacy default stream).  Calls enqueue work and
+ *     return; they do not synchronise.
+ *   - The return value is an attnw_status.  Argument errors are detected on the host and
+ *     nothing is launched.  ATTNW_ERR_TIMEOUT is only ever reported by attnw_query_status().
+ *   - Inputs must be finite.  Non-finite inputs give unspecified values in the rows they
+ *     touch and never a fault.
+ *   - Runs on the current CUDA device, which must be compute capability 10.x.  There is no
+ *     fallback path of any kind.
+ */
+#ifndef ATTNW_H_
+#define ATTNW_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum attnw_status {
+    ATTNW_OK = 0,
+    ATTNW_ERR_NULL_POINTER = 1, /* a required pointer is NULL                                   */
+    ATTNW_ERR_BAD_SHAPE = 2,    /* a size is < 1, overflows, or scale is negative / not finite  */
+    ATTNW_ERR_MISALIGNED = 3,   /* pointer not 16-byte aligned, or row pitch not 16-byte sized  */
+    ATTNW_ERR_UNSUPPORTED = 4,  /* d not in {64, 128}; device is not sm_100                     */
+    ATTNW_ERR_CUDA = 5,         /* a CUDA runtime / driver call failed (launch, map encode)     */
+    ATTNW_ERR_TIMEOUT = 6,      /* a bounded device-side wait gave up (see attnw_query_status)  */
+    ATTNW_ERR_ALIASING = 7      /* output overlaps an input in a way the kernel cannot allow    */
+} attnw_status;
+
+/*
+ * attnw_fused: P[b,h,i,j] = exp(z_ij - m_i) / sum_k exp(z_ik - m_i),
+ *              z_ij = scale * sum_c Q[b,h,i,c] * K[b,h,j,c],  m_i = max_j z_ij.
+ * (Section IV: Attention(Q,K,V) without the product with V; Section VII: n x d_k inputs,
+ *  n x n output; Eq. 1: max-subtracted Softmax over the key index j.)
+ *
+ *   Q, K   device, bfloat16, [B, H, N, d]                      (read only)
+ *   P      device, bfloat16 (attnw_fused) or float32 (attnw_fused_f32), [B, H, N, N]; every
+ *          element is written exactly once; must not overlap Q or K
+ *   B,H,N  >= 1;  N*sizeof(P element) must be a multiple of 16 (N % 8 == 0 for bfloat16,
+ *          N % 4 == 0 for float32);  d in {64, 128}
+ *   scale  finite, >= 0 (1/sqrt(d) in the paper); applied to the scores before the max
+ * Scores are accumulated in float32 on the tensor cores; max, exponentials and sums are
+ * float32; only P is rounded (to nearest even for bfloat16).
+ */
+int attnw_fused(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream);
+int attnw_fused_f32(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream);
+
+/*
+ * softmax_rows: P[i,j] = exp(S_ij - m_i) / sum_k exp(S_ik - m_i),  m_i = max_j S_ij
+ * (Softmax definition of Section VI with Eq. 1; one row is read once, kept on chip, and
+ *  written once - the "caching" form of Section VI-A - unless cols exceeds the on-chip tier,
+ *  where the exponentials are recomputed from a second read of the row.)
+ *
+ *   S      device, float32, [rows, cols]                        (read only)
+ *   P      device, bfloat16 (softmax_rows) or float32 (softmax_rows_f32), [rows, cols].
+ *          softmax_rows_f32 accepts P == S exactly (in place); any other overlap is refused
+ *   rows   >= 1;  cols >= 1 and cols % 4 == 0;  rows * cols < 2^62
+ */
+int softmax_rows(const void* S, void* P, long long rows, long long cols, void* stream);
+int softmax_rows_f32(const void* S, void* P, long long rows, long long cols, void* stream);
+
+/*
+ * The same two operations for callers whose data lives in HOST memory (Section III describes
+ * the host program's write-buffer / run / read-buffer sequence).  Pointers are HOST pointers
+ * (pinned memory gives the fastest copies; pageable memory works).  The call copies the
+ * inputs to the device, runs the kernel and copies P back, pipelined over groups of heads
+ * (or rows), and returns after the result is complete in host memory.  Device staging
+ * buffers are allocated on first use, kept per device and reused; attnw_host_release()
+ * frees them.  `p_is_f32` selects the element type of P (0 = bfloat16, 1 = float32).
+ * Not thread-safe with respect to other *_host calls on the same device.
+ */
+int attnw_fused_host(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, int p_is_f32);
+int softmax_rows_host(const void* S, void* P, long long rows, long long cols, int p_is_f32);
+int attnw_host_release(void);
+
+/*
+ * Device-side failure reporting.  Every wait inside the kernels is bounded; a wait that gives
+ * up records a code in a per-device status word, makes the kernel unwind and return normally,
+ * and the output of that launch is then undefined.  attnw_query_status() synchronises
+ * `stream`, stores the word in *device_status (0 = no failure; otherwise an implementation
+ * code naming the wait that gave up), clears it, and returns ATTNW_OK or ATTNW_ERR_TIMEOUT.
+ */
+int attnw_query_status(void* stream, unsigned int* device_status);
+
+/* Number of kernels this library has launched in the calling process since load / last reset
+ * (reset = 1 returns the count and then sets it to zero). */
+long long attnw_launch_count(int reset);
+
+/* Static string for a status code; never NULL. */
+const char* attnw_strerror(int code);
+
+/* major * 10000 + minor * 100 + patch */
+int attnw_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATTNW_H_ */

@@ -1,0 +1,378 @@
+// C ABI of libattnw.so: argument validation, tensor-map encoding and kernel launches.
+// The contract of every entry point is stated in include/attnw.h.
+#include <atomic>
+#include <climits>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <mutex>
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "../../include/attnw.h"
+#include "attnw_fused.cuh"
+#include "softmax_rows.cuh"
+
+namespace {
+
+using namespace attnw;
+
+constexpr int kMaxDevices = 64;
+constexpr int kVersion = 100;  // 0.1.0
+
+std::atomic<long long> g_launches{0};
+std::mutex g_mutex;
+
+struct DeviceInfo {
+    bool ready = false;
+    int cc_major = 0;
+    int sm_count = 0;
+    bool fused_attrs_set = false;
+};
+DeviceInfo g_devices[kMaxDevices];
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode_tiled = nullptr;
+
+// Current device's cached properties; returns an attnw_status.
+int current_device(DeviceInfo** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceInfo& d = g_devices[dev];
+    if (!d.ready) {
+        if (cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return ATTNW_ERR_CUDA;
+        }
+        d.ready = true;
+    }
+    *out = &d;
+    return d.cc_major == 10 ? ATTNW_OK : ATTNW_ERR_UNSUPPORTED;
+}
+
+int load_encoder() {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (g_encode_tiled) return ATTNW_OK;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    return ATTNW_OK;
+}
+
+// Row-major [dim2][dim1][dim0] tensor, box {box0, box1, 1}, 128-byte swizzle (box0 * esize == 128).
+int encode_3d(CUtensorMap* map, CUtensorMapDataType dtype, size_t esize, const void* base, uint64_t dim0,
+              uint64_t dim1, uint64_t dim2, uint32_t box0, uint32_t box1) {
+    const cuuint64_t dims[3] = {dim0, dim1, dim2};
+    const cuuint64_t strides[2] = {dim0 * esize, dim0 * dim1 * esize};
+    const cuuint32_t box[3] = {box0, box1, 1};
+    const cuuint32_t elem_strides[3] = {1, 1, 1};
+    CUresult r = g_encode_tiled(map, dtype, 3, const_cast<void*>(base), dims, strides, box, elem_strides,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? ATTNW_OK : ATTNW_ERR_CUDA;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool overlaps(const void* a, unsigned long long a_bytes, const void* b, unsigned long long b_bytes) {
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + b_bytes && b0 < a0 + a_bytes;
+}
+
+// Host-only checks of the fused call; no CUDA call is made here.
+int validate_fused(const void* Q, const void* K, const void* P, int B, int H, int N, int d, float scale,
+                   size_t p_esize) {
+    if (!Q || !K || !P) return ATTNW_ERR_NULL_POINTER;
+    if (B < 1 || H < 1 || N < 1 || d < 1) return ATTNW_ERR_BAD_SHAPE;
+    if (!(scale >= 0.0f) || !std::isfinite(scale)) return ATTNW_ERR_BAD_SHAPE;
+    const long long bh = static_cast<long long>(B) * H;
+    if (bh > INT_MAX) return ATTNW_ERR_BAD_SHAPE;
+    const long long ctas = bh * ((static_cast<long long>(N) + kRowsPerCta - 1) / kRowsPerCta);
+    if (ctas > INT_MAX) return ATTNW_ERR_BAD_SHAPE;
+    if (N > (1 << 24)) return ATTNW_ERR_BAD_SHAPE;  // keeps every tensor-map stride below 2^40 bytes
+    if (d != 64 && d != 128) return ATTNW_ERR_UNSUPPORTED;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(P)) return ATTNW_ERR_MISALIGNED;
+    if ((static_cast<unsigned long long>(N) * p_esize) % 16 != 0) return ATTNW_ERR_MISALIGNED;
+    if (static_cast<unsigned long long>(N) * N * p_esize >= (1ull << 40)) return ATTNW_ERR_BAD_SHAPE;
+    const unsigned long long qk_bytes = static_cast<unsigned long long>(bh) * N * d * 2ull;
+    const unsigned long long p_bytes = static_cast<unsigned long long>(bh) * N * N * p_esize;
+    if (overlaps(P, p_bytes, Q, qk_bytes) || overlaps(P, p_bytes, K, qk_bytes)) return ATTNW_ERR_ALIASING;
+    return ATTNW_OK;
+}
+
+template <int D, typename OutT>
+int launch_fused(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH, int N, float scale,
+                 cudaStream_t stream) {
+    using L = FusedSmem<D>;
+    auto kernel = attnw_fused_kernel<D, OutT>;
+    CUtensorMap tm_q, tm_k, tm_p;
+    int rc = encode_3d(&tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Q, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, K, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) {
+        if (sizeof(OutT) == 2)
+            rc = encode_3d(&tm_p, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, P, N, N, BH, 64, 32);
+        else
+            rc = encode_3d(&tm_p, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, P, N, N, BH, 32, 32);
+    }
+    if (rc != ATTNW_OK) return rc;
+    // The attribute is per device and per kernel; set it on every launch path's first use.
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    (void)dev;
+    const int row_blocks = (N + kRowsPerCta - 1) / kRowsPerCta;
+    const float scale_log2e = static_cast<float>(static_cast<double>(scale) * 1.4426950408889634074);
+    kernel<<<static_cast<unsigned>(BH * row_blocks), kFusedThreads, L::kDynamicBytes, stream>>>(tm_q, tm_k, tm_p, N,
+                                                                                                 row_blocks, scale_log2e);
+    if (cudaGetLastError() != cudaSuccess) return ATTNW_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTNW_OK;
+}
+
+template <typename OutT>
+int fused_entry(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream) {
+    int rc = validate_fused(Q, K, P, B, H, N, d, scale, sizeof(OutT));
+    if (rc != ATTNW_OK) return rc;
+    DeviceInfo* dev = nullptr;
+    rc = current_device(&dev);
+    if (rc != ATTNW_OK) return rc;
+    rc = load_encoder();
+    if (rc != ATTNW_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (d == 64) return launch_fused<64, OutT>(dev, Q, K, P, B * H, N, scale, s);
+    return launch_fused<128, OutT>(dev, Q, K, P, B * H, N, scale, s);
+}
+
+int validate_rows(const void* S, const void* P, long long rows, long long cols, size_t p_esize, bool allow_inplace) {
+    if (!S || !P) return ATTNW_ERR_NULL_POINTER;
+    if (rows < 1 || cols < 1) return ATTNW_ERR_BAD_SHAPE;
+    if (cols > (1ll << 40) || rows > (1ll << 40) || rows > (1ll << 62) / cols) return ATTNW_ERR_BAD_SHAPE;
+    if (cols % 4 != 0) return ATTNW_ERR_MISALIGNED;
+    if (!aligned16(S) || !aligned16(P)) return ATTNW_ERR_MISALIGNED;
+    const unsigned long long n = static_cast<unsigned long long>(rows) * static_cast<unsigned long long>(cols);
+    if (overlaps(S, n * 4ull, P, n * p_esize) && !(allow_inplace && S == P)) return ATTNW_ERR_ALIASING;
+    return ATTNW_OK;
+}
+
+template <typename OutT>
+int rows_entry(const void* S, void* P, long long rows, long long cols, void* stream) {
+    int rc = validate_rows(S, P, rows, cols, sizeof(OutT), sizeof(OutT) == 4);
+    if (rc != ATTNW_OK) return rc;
+    DeviceInfo* dev = nullptr;
+    rc = current_device(&dev);
+    if (rc != ATTNW_OK) return rc;
+    cudaError_t e = softmax_rows_launch<OutT>(static_cast<const float*>(S), static_cast<OutT*>(P), rows, cols,
+                                              dev->sm_count, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return ATTNW_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTNW_OK;
+}
+
+// ---- host-buffer entry points: staging buffers kept per device, two streams ---------------
+struct HostStaging {
+    void* buf[2][3] = {{nullptr, nullptr, nullptr}, {nullptr, nullptr, nullptr}};
+    size_t cap[2][3] = {{0, 0, 0}, {0, 0, 0}};
+    cudaStream_t stream[2] = {nullptr, nullptr};
+    bool streams_ready = false;
+};
+HostStaging g_staging[kMaxDevices];
+
+int staging_for_current_device(HostStaging** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ATTNW_ERR_CUDA;
+    HostStaging& st = g_staging[dev];
+    if (!st.streams_ready) {
+        for (int i = 0; i < 2; ++i)
+            if (cudaStreamCreateWithFlags(&st.stream[i], cudaStreamNonBlocking) != cudaSuccess) return ATTNW_ERR_CUDA;
+        st.streams_ready = true;
+    }
+    *out = &st;
+    return ATTNW_OK;
+}
+
+int staging_reserve(HostStaging* st, int slot, int which, size_t bytes) {
+    if (st->cap[slot][which] >= bytes) return ATTNW_OK;
+    if (st->buf[slot][which]) {
+        // The slot's stream may still be using the old buffer.
+        if (cudaStreamSynchronize(st->stream[slot]) != cudaSuccess) return ATTNW_ERR_CUDA;
+        cudaFree(st->buf[slot][which]);
+        st->buf[slot][which] = nullptr;
+        st->cap[slot][which] = 0;
+    }
+    if (cudaMalloc(&st->buf[slot][which], bytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    st->cap[slot][which] = bytes;
+    return ATTNW_OK;
+}
+
+constexpr unsigned long long kHostChunkBytes = 256ull << 20;  // target size of one staged piece of P
+
+}  // namespace
+
+extern "C" {
+
+int attnw_fused(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream) {
+    return fused_entry<__nv_bfloat16>(Q, K, P, B, H, N, d, scale, stream);
+}
+
+int attnw_fused_f32(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream) {
+    return fused_entry<float>(Q, K, P, B, H, N, d, scale, stream);
+}
+
+int softmax_rows(const void* S, void* P, long long rows, long long cols, void* stream) {
+    return rows_entry<__nv_bfloat16>(S, P, rows, cols, stream);
+}
+
+int softmax_rows_f32(const void* S, void* P, long long rows, long long cols, void* stream) {
+    return rows_entry<float>(S, P, rows, cols, stream);
+}
+
+int attnw_fused_host(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, int p_is_f32) {
+    const size_t esize = p_is_f32 ? 4 : 2;
+    if (!Q || !K || !P) return ATTNW_ERR_NULL_POINTER;
+    if (B < 1 || H < 1 || N < 1 || d < 1) return ATTNW_ERR_BAD_SHAPE;
+    if (d != 64 && d != 128) return ATTNW_ERR_UNSUPPORTED;
+    const long long bh = static_cast<long long>(B) * H;
+    if (bh > INT_MAX || N > (1 << 24)) return ATTNW_ERR_BAD_SHAPE;
+    HostStaging* st = nullptr;
+    int rc = staging_for_current_device(&st);
+    if (rc != ATTNW_OK) return rc;
+    const unsigned long long p_head = static_cast<unsigned long long>(N) * N * esize;
+    const unsigned long long qk_head = static_cast<unsigned long long>(N) * d * 2ull;
+    long long group = static_cast<long long>(kHostChunkBytes / p_head);
+    if (group < 1) group = 1;
+    if (group > bh) group = bh;
+    for (int slot = 0; slot < 2; ++slot) {
+        rc = staging_reserve(st, slot, 0, qk_head * group);
+        if (rc == ATTNW_OK) rc = staging_reserve(st, slot, 1, qk_head * group);
+        if (rc == ATTNW_OK) rc = staging_reserve(st, slot, 2, p_head * group);
+        if (rc != ATTNW_OK) return rc;
+    }
+    const char* q = static_cast<const char*>(Q);
+    const char* k = static_cast<const char*>(K);
+    char* p = static_cast<char*>(P);
+    int piece = 0;
+    for (long long h0 = 0; h0 < bh; h0 += group, ++piece) {
+        const long long g = (bh - h0 < group) ? bh - h0 : group;
+        const int slot = piece & 1;
+        cudaStream_t s = st->stream[slot];
+        if (cudaMemcpyAsync(st->buf[slot][0], q + h0 * qk_head, g * qk_head, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+            cudaMemcpyAsync(st->buf[slot][1], k + h0 * qk_head, g * qk_head, cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return ATTNW_ERR_CUDA;
+        rc = p_is_f32 ? attnw_fused_f32(st->buf[slot][0], st->buf[slot][1], st->buf[slot][2], 1, static_cast<int>(g), N,
+                                        d, scale, s)
+                      : attnw_fused(st->buf[slot][0], st->buf[slot][1], st->buf[slot][2], 1, static_cast<int>(g), N, d,
+                                    scale, s);
+        if (rc != ATTNW_OK) return rc;
+        if (cudaMemcpyAsync(p + h0 * p_head, st->buf[slot][2], g * p_head, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return ATTNW_ERR_CUDA;
+    }
+    for (int slot = 0; slot < 2; ++slot)
+        if (cudaStreamSynchronize(st->stream[slot]) != cudaSuccess) return ATTNW_ERR_CUDA;
+    return ATTNW_OK;
+}
+
+int softmax_rows_host(const void* S, void* P, long long rows, long long cols, int p_is_f32) {
+    const size_t esize = p_is_f32 ? 4 : 2;
+    if (!S || !P) return ATTNW_ERR_NULL_POINTER;
+    if (rows < 1 || cols < 1 || cols > (1ll << 40) || rows > (1ll << 40) || rows > (1ll << 62) / cols)
+        return ATTNW_ERR_BAD_SHAPE;
+    if (cols % 4 != 0) return ATTNW_ERR_MISALIGNED;
+    HostStaging* st = nullptr;
+    int rc = staging_for_current_device(&st);
+    if (rc != ATTNW_OK) return rc;
+    long long group = static_cast<long long>(kHostChunkBytes / (static_cast<unsigned long long>(cols) * 4ull));
+    if (group < 1) group = 1;
+    if (group > rows) group = rows;
+    for (int slot = 0; slot < 2; ++slot) {
+        rc = staging_reserve(st, slot, 0, static_cast<size_t>(group) * cols * 4);
+        if (rc == ATTNW_OK) rc = staging_reserve(st, slot, 2, static_cast<size_t>(group) * cols * esize);
+        if (rc != ATTNW_OK) return rc;
+    }
+    const char* src = static_cast<const char*>(S);
+    char* dst = static_cast<char*>(P);
+    int piece = 0;
+    for (long long r0 = 0; r0 < rows; r0 += group, ++piece) {
+        const long long g = (rows - r0 < group) ? rows - r0 : group;
+        const int slot = piece & 1;
+        cudaStream_t s = st->stream[slot];
+        if (cudaMemcpyAsync(st->buf[slot][0], src + r0 * cols * 4, static_cast<size_t>(g) * cols * 4,
+                            cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return ATTNW_ERR_CUDA;
+        rc = p_is_f32 ? softmax_rows_f32(st->buf[slot][0], st->buf[slot][2], g, cols, s)
+                      : softmax_rows(st->buf[slot][0], st->buf[slot][2], g, cols, s);
+        if (rc != ATTNW_OK) return rc;
+        if (cudaMemcpyAsync(dst + r0 * cols * esize, st->buf[slot][2], static_cast<size_t>(g) * cols * esize,
+                            cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return ATTNW_ERR_CUDA;
+    }
+    for (int slot = 0; slot < 2; ++slot)
+        if (cudaStreamSynchronize(st->stream[slot]) != cudaSuccess) return ATTNW_ERR_CUDA;
+    return ATTNW_OK;
+}
+
+int attnw_host_release(void) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return ATTNW_ERR_CUDA;
+    HostStaging& st = g_staging[dev];
+    for (int slot = 0; slot < 2; ++slot) {
+        if (st.streams_ready) cudaStreamSynchronize(st.stream[slot]);
+        for (int w = 0; w < 3; ++w) {
+            if (st.buf[slot][w]) cudaFree(st.buf[slot][w]);
+            st.buf[slot][w] = nullptr;
+            st.cap[slot][w] = 0;
+        }
+    }
+    return ATTNW_OK;
+}
+
+int attnw_query_status(void* stream, unsigned int* device_status) {
+    if (!device_status) return ATTNW_ERR_NULL_POINTER;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return ATTNW_ERR_CUDA;
+    unsigned int word = 0;
+    if (cudaMemcpyFromSymbol(&word, attnw::g_attnw_status, sizeof(word)) != cudaSuccess) return ATTNW_ERR_CUDA;
+    *device_status = word;
+    if (word == 0) return ATTNW_OK;
+    const unsigned int zero = 0;
+    if (cudaMemcpyToSymbol(attnw::g_attnw_status, &zero, sizeof(zero)) != cudaSuccess) return ATTNW_ERR_CUDA;
+    return ATTNW_ERR_TIMEOUT;
+}
+
+long long attnw_launch_count(int reset) {
+    return reset ? g_launches.exchange(0, std::memory_order_relaxed) : g_launches.load(std::memory_order_relaxed);
+}
+
+const char* attnw_strerror(int code) {
+    switch (code) {
+        case ATTNW_OK: return "ok";
+        case ATTNW_ERR_NULL_POINTER: return "a required pointer is NULL";
+        case ATTNW_ERR_BAD_SHAPE: return "a size is out of range, or scale is negative or not finite";
+        case ATTNW_ERR_MISALIGNED: return "a pointer or a row pitch is not a multiple of 16 bytes";
+        case ATTNW_ERR_UNSUPPORTED: return "unsupported head dimension or device (needs d in {64,128}, sm_100)";
+        case ATTNW_ERR_CUDA: return "a CUDA runtime or driver call failed";
+        case ATTNW_ERR_TIMEOUT: return "a bounded device-side wait gave up; the output of that launch is undefined";
+        case ATTNW_ERR_ALIASING: return "the output overlaps an input";
+        default: return "unknown attnw status code";
+    }
+}
+
+int attnw_version(void) { return kVersion; }
+
+}  // extern "C"

@@ -1,0 +1,215 @@
+// Dedicated row-Softmax kernels over precomputed float32 scores (Section VI, Eq. 1; the
+// B200 counterpart of the dedicated kernel of Section VI-B).
+//
+// The operation is bound by HBM traffic (4 bytes read + 2 or 4 written per element, nothing
+// to contract), so there are no tensor cores here: each row is streamed in with 128-bit
+// loads, kept in registers (the "caching" form of Section VI-A: every exponential is computed
+// once), reduced with warp shuffles (plus one shared-memory hop when a row spans several
+// warps), and written with coalesced vector stores.  Rows longer than the register tier are
+// handled by a two-read kernel that recomputes the exponentials (the "recomputing" form).
+#pragma once
+#include <cstdint>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+namespace attnw {
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+__device__ __forceinline__ float sr_ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <typename OutT>
+__device__ __forceinline__ void sr_store4(OutT* dst, float a, float b, float c, float d);
+
+template <>
+__device__ __forceinline__ void sr_store4<float>(float* dst, float a, float b, float c, float d) {
+    __stcs(reinterpret_cast<float4*>(dst), make_float4(a, b, c, d));
+}
+template <>
+__device__ __forceinline__ void sr_store4<__nv_bfloat16>(__nv_bfloat16* dst, float a, float b, float c, float d) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(c, d);
+    uint2 v;
+    v.x = *reinterpret_cast<uint32_t*>(&lo);
+    v.y = *reinterpret_cast<uint32_t*>(&hi);
+    __stcs(reinterpret_cast<uint2*>(dst), v);
+}
+
+// Reduce over the TPR threads that share a row.  TPR <= 32: shuffles inside the warp segment.
+// TPR > 32: the CTA holds exactly one row; warps exchange partials through `red`.
+template <int TPR, bool IS_MAX>
+__device__ __forceinline__ float sr_row_reduce(float v, float* red) {
+    constexpr int kShuffleSpan = TPR < 32 ? TPR : 32;
+#pragma unroll
+    for (int off = kShuffleSpan / 2; off > 0; off >>= 1) {
+        float o = __shfl_xor_sync(0xffffffffu, v, off);
+        v = IS_MAX ? fmaxf(v, o) : v + o;
+    }
+    if constexpr (TPR > 32) {
+        constexpr int kWarps = TPR / 32;
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        if (lane == 0) red[warp] = v;
+        __syncthreads();
+        float acc = red[0];
+#pragma unroll
+        for (int w = 1; w < kWarps; ++w) acc = IS_MAX ? fmaxf(acc, red[w]) : acc + red[w];
+        v = acc;
+    }
+    return v;
+}
+
+// S and P carry no __restrict__ and every load is a coherent one: the float32 variant may run
+// in place (P == S), where each thread overwrites exactly the elements it has loaded.
+//
+// Register tier: TPR threads per row, VPT float4 vectors per thread, row kept in registers.
+// A CTA has max(TPR, 256) threads and handles CTA_THREADS / TPR rows per sweep.
+template <int TPR, int VPT, typename OutT>
+__global__ void __launch_bounds__((TPR > 256 ? TPR : 256))
+softmax_rows_reg_kernel(const float* S, OutT* P, long long rows, int cols) {
+    constexpr int kThreads = TPR > 256 ? TPR : 256;
+    constexpr int kRowsPerCta = kThreads / TPR;
+    __shared__ float red_max[TPR > 32 ? TPR / 32 : 1];
+    __shared__ float red_sum[TPR > 32 ? TPR / 32 : 1];
+
+    const int nvec = cols >> 2;
+    const int sub = threadIdx.x % TPR;          // position inside the row group
+    const int row_in_cta = threadIdx.x / TPR;
+    const long long sweeps = (rows + kRowsPerCta - 1) / kRowsPerCta;
+
+    for (long long sweep = blockIdx.x; sweep < sweeps; sweep += gridDim.x) {
+        const long long row = sweep * kRowsPerCta + row_in_cta;
+        const bool row_ok = row < rows;  // uniform per row group; whole warps when TPR >= 32
+        const float4* src = reinterpret_cast<const float4*>(S + (row_ok ? row : 0) * static_cast<long long>(cols));
+        float4 v[VPT];
+        float m = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int idx = sub + k * TPR;
+            if (row_ok && idx < nvec) {
+                v[k] = __ldcs(src + idx);
+                m = fmaxf(m, fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w)));
+            } else {
+                v[k] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            }
+        }
+        m = sr_row_reduce<TPR, true>(m, red_max);
+        if (!row_ok) m = 0.0f;  // keeps the arithmetic below free of inf - inf
+        float l = 0.0f;
+        // (x - m) first: the difference is exact near the maximum, so a constant row gives exactly 1.
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            v[k].x = sr_ex2((v[k].x - m) * kLog2e);
+            v[k].y = sr_ex2((v[k].y - m) * kLog2e);
+            v[k].z = sr_ex2((v[k].z - m) * kLog2e);
+            v[k].w = sr_ex2((v[k].w - m) * kLog2e);
+            l += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+        }
+        l = sr_row_reduce<TPR, false>(l, red_sum);
+        const float inv = 1.0f / l;
+        OutT* dst = P + (row_ok ? row : 0) * static_cast<long long>(cols);
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int idx = sub + k * TPR;
+            if (row_ok && idx < nvec)
+                sr_store4<OutT>(dst + 4ll * idx, v[k].x * inv, v[k].y * inv, v[k].z * inv, v[k].w * inv);
+        }
+    }
+}
+
+// Streaming tier for rows beyond the register tier: one CTA of 1024 threads per row.  First
+// read: per-thread running maximum and sum (rescaled only when the maximum grows), merged
+// across the CTA.  Second read (mostly from L2): exponentials recomputed, normalised, stored.
+template <typename OutT>
+__global__ void __launch_bounds__(1024)
+softmax_rows_stream_kernel(const float* S, OutT* P, long long rows, long long cols) {
+    __shared__ float red_m[32];
+    __shared__ float red_l[32];
+    const long long nvec = cols >> 2;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    for (long long row = blockIdx.x; row < rows; row += gridDim.x) {
+        const float4* src = reinterpret_cast<const float4*>(S + row * cols);
+        float m = -INFINITY, l = 0.0f;
+        for (long long idx = threadIdx.x; idx < nvec; idx += 1024) {
+            const float4 x = __ldcs(src + idx);
+            const float vm = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
+            if (vm > m) {
+                l *= sr_ex2((m - vm) * kLog2e);
+                m = vm;
+            }
+            l += (sr_ex2((x.x - m) * kLog2e) + sr_ex2((x.y - m) * kLog2e)) +
+                 (sr_ex2((x.z - m) * kLog2e) + sr_ex2((x.w - m) * kLog2e));
+        }
+        // merge (m, l) pairs: inside the warp, then across warps
+        float wm = m;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) wm = fmaxf(wm, __shfl_xor_sync(0xffffffffu, wm, off));
+        float wl = (m == -INFINITY) ? 0.0f : l * sr_ex2((m - wm) * kLog2e);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) wl += __shfl_xor_sync(0xffffffffu, wl, off);
+        if (lane == 0) {
+            red_m[warp] = wm;
+            red_l[warp] = wl;
+        }
+        __syncthreads();
+        float M = red_m[0];
+#pragma unroll
+        for (int w = 1; w < 32; ++w) M = fmaxf(M, red_m[w]);
+        float L = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 32; ++w) L += (red_m[w] == -INFINITY) ? 0.0f : red_l[w] * sr_ex2((red_m[w] - M) * kLog2e);
+        __syncthreads();  // red_* are rewritten by the next row
+        const float inv = 1.0f / L;
+        OutT* dst = P + row * cols;
+        for (long long idx = threadIdx.x; idx < nvec; idx += 1024) {
+            const float4 x = __ldcs(src + idx);
+            sr_store4<OutT>(dst + 4 * idx, sr_ex2((x.x - M) * kLog2e) * inv, sr_ex2((x.y - M) * kLog2e) * inv,
+                            sr_ex2((x.z - M) * kLog2e) * inv, sr_ex2((x.w - M) * kLog2e) * inv);
+        }
+    }
+}
+
+// Host-side tier selection; returns the cudaError_t of the launch.
+template <int TPR, int VPT, typename OutT>
+inline cudaError_t sr_launch_reg(const float* S, OutT* P, long long rows, int cols, int sm_count,
+                                 cudaStream_t stream) {
+    constexpr int kThreads = TPR > 256 ? TPR : 256;
+    constexpr int kRowsPerCta = kThreads / TPR;
+    const long long sweeps = (rows + kRowsPerCta - 1) / kRowsPerCta;
+    const long long cap = static_cast<long long>(sm_count) * 64;  // enough CTAs to fill every SM several times
+    const unsigned grid = static_cast<unsigned>(sweeps < cap ? sweeps : cap);
+    softmax_rows_reg_kernel<TPR, VPT, OutT><<<grid, kThreads, 0, stream>>>(S, P, rows, cols);
+    return cudaGetLastError();
+}
+
+constexpr long long kSoftmaxRowsRegTierMaxCols = 32768;
+
+template <typename OutT>
+inline cudaError_t softmax_rows_launch(const float* S, OutT* P, long long rows, long long cols, int sm_count,
+                                       cudaStream_t stream) {
+    const long long nvec = cols / 4;
+    if (cols > kSoftmaxRowsRegTierMaxCols) {
+        const long long cap = static_cast<long long>(sm_count) * 4;
+        const unsigned grid = static_cast<unsigned>(rows < cap ? rows : cap);
+        softmax_rows_stream_kernel<OutT><<<grid, 1024, 0, stream>>>(S, P, rows, cols);
+        return cudaGetLastError();
+    }
+    const int c = static_cast<int>(cols);
+    if (nvec <= 8) return sr_launch_reg<8, 1, OutT>(S, P, rows, c, sm_count, stream);
+    if (nvec <= 16) return sr_launch_reg<8, 2, OutT>(S, P, rows, c, sm_count, stream);
+    if (nvec <= 32) return sr_launch_reg<8, 4, OutT>(S, P, rows, c, sm_count, stream);
+    if (nvec <= 64) return sr_launch_reg<32, 2, OutT>(S, P, rows, c, sm_count, stream);
+    if (nvec <= 128) return sr_launch_reg<32, 4, OutT>(S, P, rows, c, sm_count, stream);
+    if (nvec <= 256) return sr_launch_reg<32, 8, OutT>(S, P, rows, c, sm_count, stream);
+    if (nvec <= 512) return sr_launch_reg<256, 2, OutT>(S, P, rows, c, sm_count, stream);
+    if (nvec <= 1024) return sr_launch_reg<256, 4, OutT>(S, P, rows, c, sm_count, stream);
+    if (nvec <= 2048) return sr_launch_reg<256, 8, OutT>(S, P, rows, c, sm_count, stream);
+    if (nvec <= 4096) return sr_launch_reg<1024, 4, OutT>(S, P, rows, c, sm_count, stream);
+    return sr_launch_reg<1024, 8, OutT>(S, P, rows, c, sm_count, stream);
+}
+
+}  // namespace attnw
