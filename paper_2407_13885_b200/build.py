@@ -25,6 +25,9 @@ def nvcc_command(out: str, verbose_ptxas: bool = False) -> list[str]:
            "-shared", "-Xcompiler", "-fPIC", "-o", out, *SOURCES]
     if verbose_ptxas:
         cmd[1:1] = ["-Xptxas", "-v"]
+    # Extra -D definitions for experiments and debug builds, e.g. ATTNW_DEFINES="ATTNW_TIMELINE=700".
+    for d in os.environ.get("ATTNW_DEFINES", "").split():
+        cmd.insert(1, "-D" + d)
     return cmd
 
 

@@ -124,9 +124,9 @@ int launch_fused(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH,
     if (rc == ATTNW_OK) rc = encode_3d(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, K, D, N, BH, 64, kTile);
     if (rc == ATTNW_OK) {
         if (sizeof(OutT) == 2)
-            rc = encode_3d(&tm_p, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, P, N, N, BH, 64, 32);
+            rc = encode_3d(&tm_p, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, P, N, N, BH, 64, kTile);
         else
-            rc = encode_3d(&tm_p, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, P, N, N, BH, 32, 32);
+            rc = encode_3d(&tm_p, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, P, N, N, BH, 32, kTile);
     }
     if (rc != ATTNW_OK) return rc;
     // The attribute is per device and per kernel; set it on every launch path's first use.
@@ -374,5 +374,21 @@ const char* attnw_strerror(int code) {
 }
 
 int attnw_version(void) { return kVersion; }
+#ifdef ATTNW_CTA_CLOCK
+// Debug builds only (-DATTNW_CTA_CLOCK): per-CTA cycle and nanosecond spans of the last fused launch.
+int attnw_debug_cta_clock(long long* out) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return ATTNW_ERR_CUDA;
+    return cudaMemcpyFromSymbol(out, attnw::g_attnw_cta_clock, sizeof(long long) * 4096 * 4) == cudaSuccess ? ATTNW_OK
+                                                                                                           : ATTNW_ERR_CUDA;
+}
+#endif
+#ifdef ATTNW_TIMELINE
+// Debug builds only (-DATTNW_TIMELINE=<cta index>): copies the cycle stamps of that CTA to the host.
+int attnw_debug_timeline(long long* out) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return ATTNW_ERR_CUDA;
+    return cudaMemcpyFromSymbol(out, attnw::g_attnw_timeline, sizeof(long long) * 16 * 160) == cudaSuccess ? ATTNW_OK
+                                                                                                          : ATTNW_ERR_CUDA;
+}
+#endif
 
 }  // extern "C"
