@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/; None until a capture exists for that kernel.
-NCU_TRAFFIC_BYTES = {"c3": None, "c4": None}
+NCU_TRAFFIC_BYTES = {"c3": 8 * (34.04e6 + 478.30e6), "c4": 4 * (268.45e6 + 98.18e6)}
 
 
 def load_peaks():
