@@ -58,6 +58,17 @@ int attnw_fused(const void* Q, const void* K, void* P, int B, int H, int N, int 
 int attnw_fused_f32(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream);
 
 /*
+ * Which kernel attnw_fused uses (process-wide; the results are the same within the stated tolerances):
+ *   0  choose by measurement (default): at present the two-pass kernel for every shape
+ *   1  two-pass kernel: statistics pass + normalise pass that recomputes the score tiles; any N
+ *   2  SRAM-resident kernel: a cluster of ceil(N/512) CTAs keeps a 128-row block of scores in tensor
+ *      memory and exchanges local row maxima and sums across CTAs, as the fused kernel of Section VII
+ *      does across Tensix cores; a call it cannot serve then returns ATTNW_ERR_UNSUPPORTED
+ * Returns ATTNW_ERR_BAD_SHAPE for any other value.
+ */
+int attnw_set_fused_variant(int variant);
+
+/*
  * softmax_rows: P[i,j] = exp(S_ij - m_i) / sum_k exp(S_ik - m_i),  m_i = max_j S_ij
  * (Softmax definition of Section VI with Eq. 1; one row is read once, kept on chip, and
  *  written once - the "caching" form of Section VI-A - unless cols exceeds the on-chip tier,

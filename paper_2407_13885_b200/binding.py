@@ -25,6 +25,7 @@ SIGNATURES = {
     "softmax_rows_host": (_int, [_vp, _vp, _ll, _ll, _int]),
     "attnw_host_release": (_int, []),
     "attnw_query_status": (_int, [_vp, ctypes.POINTER(ctypes.c_uint)]),
+    "attnw_set_fused_variant": (_int, [_int]),
     "attnw_launch_count": (_ll, [_int]),
     "attnw_strerror": (ctypes.c_char_p, [_int]),
     "attnw_version": (_int, []),
@@ -64,6 +65,15 @@ def strerror(code: int) -> str:
 
 def version() -> int:
     return int(lib.attnw_version())
+
+
+FUSED_VARIANTS = {"auto": 0, "two_pass": 1, "resident": 2}
+
+
+def set_fused_variant(variant: str | int) -> None:
+    """Selects the kernel behind ``attnw_fused``: "auto" (by shape), "two_pass" or "resident"."""
+    code = FUSED_VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    _check(lib.attnw_set_fused_variant(code), "attnw_set_fused_variant")
 
 
 def launch_count(reset: bool = False) -> int:

@@ -13,6 +13,7 @@
 
 #include "../../include/attnw.h"
 #include "attnw_fused.cuh"
+#include "attnw_resident.cuh"
 #include "softmax_rows.cuh"
 
 namespace {
@@ -23,6 +24,7 @@ constexpr int kMaxDevices = 64;
 constexpr int kVersion = 100;  // 0.1.0
 
 std::atomic<long long> g_launches{0};
+std::atomic<int> g_fused_variant{0};  // 0 = choose by shape, 1 = two-pass, 2 = SRAM-resident
 std::mutex g_mutex;
 
 struct DeviceInfo {
@@ -144,6 +146,55 @@ int launch_fused(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH,
     return ATTNW_OK;
 }
 
+// SRAM-resident single-pass kernel: one cluster of ceil(N / 512) CTAs per 128-row block, persistent over
+// units of work.  Returns ATTNW_ERR_UNSUPPORTED when the device cannot co-schedule such a cluster.
+template <int D>
+int launch_resident(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH, int N, float scale,
+                    cudaStream_t stream) {
+    using L = ResidentSmem<D>;
+    auto kernel = attnw_resident_kernel<D>;
+    CUtensorMap tm_q, tm_k, tm_p;
+    int rc = encode_3d(&tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Q, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, K, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_p, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, P, N, N, BH, 64, kTile);
+    if (rc != ATTNW_OK) return rc;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    const int cluster_ctas = (N + kSlab - 1) / kSlab;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(cluster_ctas);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kResidentThreads, 1, 1);
+    cfg.dynamicSmemBytes = L::kDynamicBytes;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cfg.gridDim = dim3(static_cast<unsigned>(cluster_ctas * dev->sm_count), 1, 1);
+    int max_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg) != cudaSuccess || max_clusters < 1) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_UNSUPPORTED;
+    }
+    const int row_blocks = (N + kTile - 1) / kTile;
+    const long long total_items = static_cast<long long>(BH) * row_blocks;
+    if (total_items > INT_MAX) return ATTNW_ERR_BAD_SHAPE;
+    const int clusters = total_items < max_clusters ? static_cast<int>(total_items) : max_clusters;
+    cfg.gridDim = dim3(static_cast<unsigned>(clusters * cluster_ctas), 1, 1);
+    const float scale_log2e = static_cast<float>(static_cast<double>(scale) * 1.4426950408889634074);
+    if (cudaLaunchKernelEx(&cfg, kernel, tm_q, tm_k, tm_p, N, static_cast<int>(total_items), cluster_ctas, scale_log2e) !=
+        cudaSuccess) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTNW_OK;
+}
+
 template <typename OutT>
 int fused_entry(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream) {
     int rc = validate_fused(Q, K, P, B, H, N, d, scale, sizeof(OutT));
@@ -154,6 +205,14 @@ int fused_entry(const void* Q, const void* K, void* P, int B, int H, int N, int 
     rc = load_encoder();
     if (rc != ATTNW_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int variant = g_fused_variant.load(std::memory_order_relaxed);
+    const bool resident_fits = sizeof(OutT) == 2 && N <= kResidentMaxN;
+    if (variant == 2 && !resident_fits) return ATTNW_ERR_UNSUPPORTED;
+    if (resident_fits && variant == 2) {
+        rc = (d == 64) ? launch_resident<64>(dev, Q, K, P, B * H, N, scale, s)
+                       : launch_resident<128>(dev, Q, K, P, B * H, N, scale, s);
+        if (rc != ATTNW_ERR_UNSUPPORTED || variant == 2) return rc;  // no cluster of that size here: two-pass
+    }
     if (d == 64) return launch_fused<64, OutT>(dev, Q, K, P, B * H, N, scale, s);
     return launch_fused<128, OutT>(dev, Q, K, P, B * H, N, scale, s);
 }
@@ -353,6 +412,12 @@ int attnw_query_status(void* stream, unsigned int* device_status) {
     const unsigned int zero = 0;
     if (cudaMemcpyToSymbol(attnw::g_attnw_status, &zero, sizeof(zero)) != cudaSuccess) return ATTNW_ERR_CUDA;
     return ATTNW_ERR_TIMEOUT;
+}
+
+int attnw_set_fused_variant(int variant) {
+    if (variant < 0 || variant > 2) return ATTNW_ERR_BAD_SHAPE;
+    g_fused_variant.store(variant, std::memory_order_relaxed);
+    return ATTNW_OK;
 }
 
 long long attnw_launch_count(int reset) {

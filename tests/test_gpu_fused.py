@@ -19,11 +19,15 @@ def attnw():
     return binding
 
 
-def run_fused(attnw, q_bits, k_bits, scale, dtype):
+def run_fused(attnw, q_bits, k_bits, scale, dtype, variant="auto"):
     B, H, N, d = q_bits.shape
     raw, P, g = guarded_empty((B, H, N, N), dtype)
-    attnw.attnw_fused(bits_to_cuda_bf16(q_bits), bits_to_cuda_bf16(k_bits), scale, P=P)
-    torch.cuda.synchronize()
+    attnw.set_fused_variant(variant)
+    try:
+        attnw.attnw_fused(bits_to_cuda_bf16(q_bits), bits_to_cuda_bf16(k_bits), scale, P=P)
+        torch.cuda.synchronize()
+    finally:
+        attnw.set_fused_variant("auto")
     assert attnw.query_status() == 0
     assert_guards_intact(raw, g)
     return P
@@ -42,6 +46,71 @@ def test_fused_matches_oracle(attnw, B, H, N, d, dtype):
     scale = float(np.float32(1.0 / math.sqrt(d)))
     P = run_fused(attnw, q, k, scale, dtype)
     assert_close_to_oracle(P, oracle.attnw(q, k, scale), f"B{B} H{H} N{N} d{d}")
+
+
+# The SRAM-resident cluster kernel: cluster sizes 1..8, ragged slabs, a last CTA with one to four slots in use.
+RESIDENT_SHAPES = [(1, 1, 128, 64), (1, 1, 512, 128), (1, 2, 1024, 128), (1, 3, 384, 64), (2, 2, 2048, 64),
+                   (1, 2, 4096, 128), (1, 1, 200, 128), (1, 1, 1160, 64), (1, 2, 2568, 128), (1, 1, 8, 64),
+                   (1, 1, 3080, 64), (3, 5, 640, 128)]
+
+
+@pytest.mark.parametrize("B,H,N,d", RESIDENT_SHAPES)
+def test_resident_variant_matches_oracle(attnw, B, H, N, d):
+    q, k = small_fused_inputs(B, H, N, d, stream=N + d + 7)
+    scale = float(np.float32(1.0 / math.sqrt(d)))
+    P = run_fused(attnw, q, k, scale, torch.bfloat16, variant="resident")
+    assert_close_to_oracle(P, oracle.attnw(q, k, scale), f"resident B{B} H{H} N{N} d{d}")
+
+
+def test_resident_variant_large_logits_and_limits(attnw):
+    q, k = small_fused_inputs(1, 2, 2048, 128, sigma=4.0, stream=56)
+    scale = float(np.float32(1.0 / math.sqrt(128.0)))
+    ref = oracle.attnw(q, k, scale)
+    assert ref.max() > 0.9
+    assert_close_to_oracle(run_fused(attnw, q, k, scale, torch.bfloat16, variant="resident"), ref, "resident sigma 4")
+    # identical keys: exactly uniform after rounding to bf16
+    key = inputs.normal_bf16_bits(3, 3, 128, 1.0)
+    kk = np.broadcast_to(key, (1, 2, 2048, 128)).copy()
+    P = run_fused(attnw, q, kk, 0.3, torch.bfloat16, variant="resident")
+    assert bool((P == 1.0 / 2048).all())
+    # beyond its range, or for float32 output, the resident kernel refuses instead of silently switching
+    big = torch.zeros((1, 1, 4104, 64), dtype=torch.bfloat16, device="cuda")
+    attnw.set_fused_variant("resident")
+    try:
+        with pytest.raises(attnw.AttnwError) as e:
+            attnw.attnw_fused(big, big, 0.1)
+        assert e.value.code == 4
+        small = torch.zeros((1, 1, 128, 64), dtype=torch.bfloat16, device="cuda")
+        with pytest.raises(attnw.AttnwError) as e:
+            attnw.attnw_fused(small, small, 0.1, out_dtype=torch.float32)
+        assert e.value.code == 4
+    finally:
+        attnw.set_fused_variant("auto")
+
+
+def test_resident_variant_full_size_c3_sampled(attnw):
+    w = inputs.WORKLOADS["c3"]
+    q, k = inputs.make_qk(w)
+    q = q.reshape(w.B, w.H, w.N, w.d)
+    k = k.reshape(w.B, w.H, w.N, w.d)
+    P = torch.empty((w.B, w.H, w.N, w.N), dtype=torch.bfloat16, device="cuda")
+    P.view(torch.int16).fill_(-1)
+    attnw.set_fused_variant("resident")
+    try:
+        attnw.attnw_fused(bits_to_cuda_bf16(q), bits_to_cuda_bf16(k), w.scale, P=P)
+        torch.cuda.synchronize()
+    finally:
+        attnw.set_fused_variant("auto")
+    assert attnw.query_status() == 0
+    flat = P.view(w.B * w.H, w.N, w.N)
+    for bh in range(w.B * w.H):
+        head = flat[bh]
+        assert not bool(torch.isnan(head).any()), f"unwritten or NaN element in head {bh}"
+        assert float((head.to(torch.float64).sum(-1) - 1.0).abs().max()) <= TOL[torch.bfloat16]["rowsum"]
+    ids = sample_rows(w)
+    ref = oracle.attnw_rows(q, k, w.scale, ids)
+    got = to_f64(P.view(-1, w.N)[torch.from_numpy(ids).cuda()])
+    assert float(np.max(np.abs(got - ref))) <= TOL[torch.bfloat16]["abs"]
 
 
 @pytest.mark.parametrize("N", [132, 260, 1004])
