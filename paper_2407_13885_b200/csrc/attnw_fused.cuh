@@ -20,8 +20,9 @@
 // staging and TMA stores (full 128-byte lines; ragged edges clipped by the tensor map).
 //
 // The exponentials dominate the arithmetic (2 per element against 16 MUFU results per clock
-// per SM), so a fixed share of them is evaluated on the FMA pipes instead: Cody-Waite range
-// reduction and a cubic minimax polynomial, in packed two-wide fp32 instructions.
+// per SM).  A share of them can be evaluated on the FMA pipes instead (Cody-Waite range
+// reduction and a cubic minimax polynomial, in packed two-wide fp32 instructions); see
+// ATTNW_POLY_PAIRS_* below for why that share is zero by default.
 #pragma once
 #include <cstdint>
 #include <cuda.h>
@@ -66,12 +67,15 @@ constexpr int kStageBoxBytes = 32 * 128;  // one staged store box: 32 rows x 128
 constexpr long long kWaitLimitCycles = 2000000000ll;  // about one second
 
 // Of every 8 consecutive column pairs, this many take the polynomial path (bf16 output only;
-// the float32 variant keeps every exponential on the MUFU for accuracy).
+// the float32 variant keeps every exponential on the MUFU for accuracy).  Default 0: measured on
+// B200, the kernel is bound by per-warp latency and, in a sustained loop, by the power the two
+// tensor-core passes draw - not by MUFU throughput - so moving exponentials to the FMA pipes
+// (tried at 2/8 .. 5/8) changes nothing or costs time.  Kept as a build-time knob.
 #ifndef ATTNW_POLY_PAIRS_STATS
-#define ATTNW_POLY_PAIRS_STATS 3
+#define ATTNW_POLY_PAIRS_STATS 0
 #endif
 #ifndef ATTNW_POLY_PAIRS_NORM
-#define ATTNW_POLY_PAIRS_NORM 3
+#define ATTNW_POLY_PAIRS_NORM 0
 #endif
 
 enum : uint32_t {  // which wait gave up (low byte of the status word)
@@ -186,12 +190,8 @@ __device__ __forceinline__ float sum_exp2_chunk(const float (&s)[kChunk], uint64
         } else {
             float x0, x1;
             ptx::unpack2(x2, x0, x1);
-#ifdef ATTNW_X_NOEXP
-            e0 = x0; e1 = x1;
-#else
             e0 = ptx::ex2_approx(x0);
             e1 = ptx::ex2_approx(x1);
-#endif
         }
         if (RAGGED) {  // masked columns contribute nothing, also when c2 == 0
             e0 = (j + 0 < valid) ? e0 : 0.f;
@@ -462,6 +462,7 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const bool issuer = quarter == 0;
             const int out_row = row0 + q * kTile;  // first row of the group's boxes (always inside P)
             const uint32_t sw = static_cast<uint32_t>(lane & 7);
+            const uint32_t row_sw = my_row + (sw << 4);  // 16-byte piece g of the row lives at row_sw ^ (g << 4)
             const uint64_t stream_out = ptx::policy_evict_first();
             const uint64_t nshift2 = ptx::pack2(-shift, -shift);
             for (int it = T; ok && it < total_iters; ++it) {
@@ -504,12 +505,8 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         } else {
                             float x0, x1;
                             ptx::unpack2(x2, x0, x1);
-#ifdef ATTNW_X_NOEXP
-                            s[j] = x0; s[j + 1] = x1;
-#else
                             s[j] = ptx::ex2_approx(x0);
                             s[j + 1] = ptx::ex2_approx(x1);
-#endif
                         }
                         if constexpr (!kBf16Out) {
                             s[j] *= inv_l;
@@ -520,7 +517,7 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         // this chunk is 64 bytes of the thread's 128-byte staging row: 16-byte pieces 4c .. 4c+3
 #pragma unroll
                         for (int g = 0; g < 4; ++g)
-                            ptx::st_shared_v4(my_row + ((static_cast<uint32_t>(c * 4 + g) ^ sw) << 4),
+                            ptx::st_shared_v4(row_sw ^ (static_cast<uint32_t>(c * 4 + g) << 4),
                                               ptx::pack_bf16x2(s[g * 8 + 0], s[g * 8 + 1]),
                                               ptx::pack_bf16x2(s[g * 8 + 2], s[g * 8 + 3]),
                                               ptx::pack_bf16x2(s[g * 8 + 4], s[g * 8 + 5]),
@@ -554,11 +551,7 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                                                                 kSiteStageFilled));
                         if (!ok) break;
                         const int out_col = kt * kTile + half * kHalf + (kBf16Out ? 0 : c * kChunk);
-#ifdef ATTNW_X_NOSTORE
-                        if (lane == 0 && out_col < N && s[0] == 12345.f) {
-#else
                         if (lane == 0 && out_col < N) {
-#endif
                             ptx::tma_store_3d(&tm_p, gbuf, out_col, out_row, bh, stream_out);
                             ptx::bulk_commit_group();
                         }
