@@ -37,7 +37,8 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/; None until a capture exists for that kernel.
-NCU_TRAFFIC_BYTES = {"c3": 8 * (34.04e6 + 478.30e6), "c4": 4 * (268.45e6 + 98.18e6)}
+NCU_TRAFFIC_BYTES = {"c3": 8 * (33.64e6 + 476.31e6), "c3_two_pass": 8 * (33.97e6 + 477.69e6),
+                     "c4": 4 * (268.45e6 + 98.18e6)}
 
 
 def load_peaks():
@@ -248,6 +249,7 @@ def run_profile_case(args):
     import torch
     from paper_2407_13885_b200 import binding, inputs
     torch.cuda.set_device(0)
+    binding.set_fused_variant(args.variant)
     if args.profile == "fused":
         base = inputs.WORKLOADS[args.workload]
         heads = max(1, min(base.B * base.H, (512 << 20) // (base.N * base.N * 2)))
@@ -290,6 +292,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     w = inputs.WORKLOADS[args.workload]
     peaks = load_peaks()
+    binding.set_fused_variant(args.variant)
 
     # seeded inputs: every rank draws its own replica of the workload (weak scaling)
     q, k = inputs.make_qk(w, seed=inputs.SEED + rank)
@@ -375,13 +378,15 @@ def run_ours(args):
     t_hbm = bytes_alg / (peaks["hbm_gbs"] * 1e9)
     t_flop = w.flops / (peaks["bf16_tflops"] * 1e12)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                "frac": achieved / peaks["hbm_gbs"],
+                "traffic": NCU_TRAFFIC_BYTES.get(w.name + ("_two_pass" if args.variant == "two_pass" else "")),
                 "peak_source": f"of {peaks['source']}",
                 "algorithmic_bytes_per_launch": bytes_alg,
                 "roofline_time_us": 1e6 * max(t_hbm, t_flop), "kernel_time_us": 1e6 * kernel_s,
                 "time_frac_of_roofline": max(t_hbm, t_flop) / kernel_s,
                 "tensor_time_us_at_burst_peak": 1e6 * t_flop,
-                "kernel": "attnw_fused_kernel<128, bf16>"}
+                "kernel": "attnw_fused_kernel<128, bf16> (two-pass)" if (args.variant == "two_pass" or w.N > 4096)
+                else "attnw_resident_kernel<128> (SRAM-resident, clusters of %d)" % ((w.N + 511) // 512)}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -436,6 +441,8 @@ def main():
     ap.add_argument("--no-secondary", action="store_true")
     ap.add_argument("--no-sustained", action="store_true")
     ap.add_argument("--sustained-seconds", type=float, default=2.0)
+    ap.add_argument("--variant", choices=["auto", "two_pass", "resident"], default="auto",
+                    help="kernel behind attnw_fused (see attnw_set_fused_variant)")
     ap.add_argument("--profile", choices=["fused", "rows"], default=None,
                     help="run a reduced case of one kernel for an ncu capture instead of the benchmark")
     args = ap.parse_args()

@@ -208,7 +208,13 @@ int fused_entry(const void* Q, const void* K, void* P, int B, int H, int N, int 
     const int variant = g_fused_variant.load(std::memory_order_relaxed);
     const bool resident_fits = sizeof(OutT) == 2 && N <= kResidentMaxN;
     if (variant == 2 && !resident_fits) return ATTNW_ERR_UNSUPPORTED;
-    if (resident_fits && variant == 2) {
+    // Choice by shape: the resident kernel wins once every cluster has a long list of row blocks to walk
+    // (measured: 1.46 vs 1.52 ms at B*H = 128, N = 4096, d = 128); with few row blocks per cluster its
+    // set-up and its exchange latency are not amortised (0.057 vs 0.049 ms at B*H = 12, N = 2048, d = 64).
+    const long long row_blocks = static_cast<long long>(B) * H * ((N + kTile - 1) / kTile);
+    const long long clusters_at_most = dev->sm_count / ((N + kSlab - 1) / kSlab);
+    const bool resident_pays = row_blocks >= 32 * clusters_at_most;
+    if (resident_fits && (variant == 2 || (variant == 0 && resident_pays))) {
         rc = (d == 64) ? launch_resident<64>(dev, Q, K, P, B * H, N, scale, s)
                        : launch_resident<128>(dev, Q, K, P, B * H, N, scale, s);
         if (rc != ATTNW_ERR_UNSUPPORTED || variant == 2) return rc;  // no cluster of that size here: two-pass
