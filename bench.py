@@ -386,7 +386,9 @@ def run_ours(args):
                 "time_frac_of_roofline": max(t_hbm, t_flop) / kernel_s,
                 "tensor_time_us_at_burst_peak": 1e6 * t_flop,
                 "kernel": "attnw_fused_kernel<128, bf16> (two-pass)" if (args.variant == "two_pass" or w.N > 4096)
-                else "attnw_resident_kernel<128> (SRAM-resident, clusters of %d)" % ((w.N + 511) // 512)}
+                else ("attnw_resident_kernel<128> (SRAM-resident, clusters of %d)" % ((w.N + 511) // 512)
+                      + (" on the SMs clusters can occupy + attnw_fused_kernel<128, bf16> on the rest: one split launch per step"
+                         if args.variant == "auto" else ""))}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,

@@ -61,7 +61,10 @@ int attnw_fused_f32(const void* Q, const void* K, void* P, int B, int H, int N, 
  * Which kernel attnw_fused uses (process-wide; the results are the same within the stated tolerances):
  *   0  choose by shape (default): the SRAM-resident kernel when P is bfloat16, N <= 4096 and every
  *      cluster has at least 32 row blocks of 128 queries to walk; the two-pass kernel otherwise
- *      (and always for attnw_fused_f32)
+ *      (and always for attnw_fused_f32).  Clusters of 8 cannot occupy every SM, so such a call is
+ *      split: most heads go to the resident kernel on `stream`, the rest to the two-pass kernel on a
+ *      per-device side stream that forks from and joins `stream` with events (first use creates the
+ *      side stream and two events); work enqueued on `stream` afterwards sees the whole result.
  *   1  two-pass kernel: statistics pass + normalise pass that recomputes the score tiles; any N
  *   2  SRAM-resident kernel: a cluster of ceil(N/512) CTAs keeps a 128-row block of scores in tensor
  *      memory and exchanges local row maxima and sums across CTAs, as the fused kernel of Section VII

@@ -25,14 +25,19 @@ constexpr int kVersion = 100;  // 0.1.0
 
 std::atomic<long long> g_launches{0};
 std::atomic<int> g_fused_variant{0};  // 0 = choose by shape, 1 = two-pass, 2 = SRAM-resident
+constexpr double kTwoPassPerSm = 0.9;  // measured: per-SM throughput of the two-pass kernel relative to the resident one
 std::mutex g_mutex;
 
 struct DeviceInfo {
     bool ready = false;
     int cc_major = 0;
     int sm_count = 0;
-    bool fused_attrs_set = false;
+    int resident_clusters[2][kMaxClusterCtas + 1] = {};  // [d == 128][cluster size]: co-resident clusters, 0 = not asked yet
+    // fork/join objects for launches that split a call over two kernels (created on first use)
+    cudaStream_t side_stream = nullptr;
+    cudaEvent_t fork_event = nullptr, join_event = nullptr;
 };
+std::mutex g_split_mutex;
 DeviceInfo g_devices[kMaxDevices];
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -146,8 +151,38 @@ int launch_fused(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH,
     return ATTNW_OK;
 }
 
+// How many clusters of `cluster_ctas` CTAs of the resident kernel the device can hold at once (cached).
+template <int D>
+int resident_max_clusters(DeviceInfo* dev, int cluster_ctas) {
+    int& cached = dev->resident_clusters[D == 128 ? 1 : 0][cluster_ctas];
+    if (cached != 0) return cached;
+    using L = ResidentSmem<D>;
+    auto kernel = attnw_resident_kernel<D>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return cached = -1;
+    }
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(cluster_ctas);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kResidentThreads, 1, 1);
+    cfg.dynamicSmemBytes = L::kDynamicBytes;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cfg.gridDim = dim3(static_cast<unsigned>(cluster_ctas * dev->sm_count), 1, 1);
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n < 1) {
+        (void)cudaGetLastError();
+        n = -1;
+    }
+    return cached = n;
+}
+
 // SRAM-resident single-pass kernel: one cluster of ceil(N / 512) CTAs per 128-row block, persistent over
-// units of work.  Returns ATTNW_ERR_UNSUPPORTED when the device cannot co-schedule such a cluster.
+// a list of row blocks.  Returns ATTNW_ERR_UNSUPPORTED when the device cannot co-schedule such a cluster.
 template <int D>
 int launch_resident(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH, int N, float scale,
                     cudaStream_t stream) {
@@ -174,12 +209,8 @@ int launch_resident(DeviceInfo* dev, const void* Q, const void* K, void* P, int 
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cfg.gridDim = dim3(static_cast<unsigned>(cluster_ctas * dev->sm_count), 1, 1);
-    int max_clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg) != cudaSuccess || max_clusters < 1) {
-        (void)cudaGetLastError();
-        return ATTNW_ERR_UNSUPPORTED;
-    }
+    const int max_clusters = resident_max_clusters<D>(dev, cluster_ctas);
+    if (max_clusters < 1) return ATTNW_ERR_UNSUPPORTED;
     const int row_blocks = (N + kTile - 1) / kTile;
     const long long total_items = static_cast<long long>(BH) * row_blocks;
     if (total_items > INT_MAX) return ATTNW_ERR_BAD_SHAPE;
@@ -215,6 +246,63 @@ int fused_entry(const void* Q, const void* K, void* P, int B, int H, int N, int 
     const long long clusters_at_most = dev->sm_count / ((N + kSlab - 1) / kSlab);
     const bool resident_pays = row_blocks >= 32 * clusters_at_most;
     if (resident_fits && (variant == 2 || (variant == 0 && resident_pays))) {
+        if constexpr (sizeof(OutT) == 2) {
+            // Clusters of 8 cannot occupy every SM (15 x 8 = 120 of 148 on B200).  When the call is chosen by
+            // shape, the heads are split: the resident kernel takes most of them on the caller's stream, and
+            // the two-pass kernel, forked onto a side stream, works through the rest on the SMs the clusters
+            // leave idle; the caller's stream joins before the call's work counts as done.
+            const int cluster_ctas = (N + kSlab - 1) / kSlab;
+            const int clusters = (d == 64) ? resident_max_clusters<64>(dev, cluster_ctas)
+                                           : resident_max_clusters<128>(dev, cluster_ctas);
+            const int bh = B * H;
+            const int idle_sms = clusters > 0 ? dev->sm_count - clusters * cluster_ctas : 0;
+            int bh_two_pass = 0;
+            if (variant == 0 && idle_sms >= 8 && bh >= 8) {
+                // Cost model in units of one resident row block: a cluster finishes one row block per unit, a
+                // two-pass CTA (256 rows on one SM) takes 2 * C / kTwoPassPerSm units, both in whole waves.
+                const long long blocks_per_head = (N + kTile - 1) / kTile;
+                const long long ctas_per_head = (N + kRowsPerCta - 1) / kRowsPerCta;
+                const double cta_units = 2.0 * cluster_ctas / kTwoPassPerSm;
+                double best = static_cast<double>((bh * blocks_per_head + clusters - 1) / clusters);
+                for (int cand = 1; cand <= bh / 2; ++cand) {
+                    const double t_res = static_cast<double>(((bh - cand) * blocks_per_head + clusters - 1) / clusters);
+                    const double t_two = static_cast<double>((cand * ctas_per_head + idle_sms - 1) / idle_sms) * cta_units;
+                    const double t = t_res > t_two ? t_res : t_two;
+                    if (t < best) {
+                        best = t;
+                        bh_two_pass = cand;
+                    }
+                }
+            }
+            if (bh_two_pass > 0) {
+                std::lock_guard<std::mutex> lock(g_split_mutex);
+                if (!dev->side_stream) {
+                    if (cudaStreamCreateWithFlags(&dev->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+                        cudaEventCreateWithFlags(&dev->fork_event, cudaEventDisableTiming) != cudaSuccess ||
+                        cudaEventCreateWithFlags(&dev->join_event, cudaEventDisableTiming) != cudaSuccess) {
+                        (void)cudaGetLastError();
+                        return ATTNW_ERR_CUDA;
+                    }
+                }
+                const int bh_res = bh - bh_two_pass;
+                const size_t qk_off = static_cast<size_t>(bh_res) * N * d * 2;
+                const size_t p_off = static_cast<size_t>(bh_res) * N * N * 2;
+                const char* q2 = static_cast<const char*>(Q) + qk_off;
+                const char* k2 = static_cast<const char*>(K) + qk_off;
+                char* p2 = static_cast<char*>(P) + p_off;
+                if (cudaEventRecord(dev->fork_event, s) != cudaSuccess) return ATTNW_ERR_CUDA;
+                rc = (d == 64) ? launch_resident<64>(dev, Q, K, P, bh_res, N, scale, s)
+                               : launch_resident<128>(dev, Q, K, P, bh_res, N, scale, s);
+                if (rc != ATTNW_OK) return rc;
+                if (cudaStreamWaitEvent(dev->side_stream, dev->fork_event, 0) != cudaSuccess) return ATTNW_ERR_CUDA;
+                rc = (d == 64) ? launch_fused<64, OutT>(dev, q2, k2, p2, bh_two_pass, N, scale, dev->side_stream)
+                               : launch_fused<128, OutT>(dev, q2, k2, p2, bh_two_pass, N, scale, dev->side_stream);
+                if (cudaEventRecord(dev->join_event, dev->side_stream) != cudaSuccess ||
+                    cudaStreamWaitEvent(s, dev->join_event, 0) != cudaSuccess)
+                    return ATTNW_ERR_CUDA;
+                return rc;
+            }
+        }
         rc = (d == 64) ? launch_resident<64>(dev, Q, K, P, B * H, N, scale, s)
                        : launch_resident<128>(dev, Q, K, P, B * H, N, scale, s);
         if (rc != ATTNW_ERR_UNSUPPORTED || variant == 2) return rc;  // no cluster of that size here: two-pass
