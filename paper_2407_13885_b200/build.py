@@ -9,7 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libattnw.so")
 SOURCES = [os.path.join(_CSRC, "attnw_api.cu")]
-_DEPS = [os.path.join(_CSRC, f) for f in ("attnw_api.cu", "attnw_fused.cuh", "softmax_rows.cuh", "ptx.cuh")] + [
+_DEPS = [os.path.join(_CSRC, f) for f in sorted(os.listdir(_CSRC))] + [
     os.path.join(os.path.dirname(_PKG), "include", "attnw.h")]
 
 

@@ -373,7 +373,7 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const float c2 = scale_log2e;
             const uint64_t c2c2 = ptx::pack2(c2, c2);
             float smax = -3.0e38f;   // running maximum of the raw scores this thread has seen
-            float mb = smax * c2;    // the offset the exponentials in l are relative to: fl(smax * c2)
+            float mb = smax;         // the offset the exponentials in l are relative to: fl(smax * c2), finite from the start
             float l = 0.0f;          // running sum of 2^(c2 * s - mb) over this thread's columns
             bool ok = true;
             const bool stamp = (warp & 7) == 0 && lane == 0;
@@ -420,7 +420,7 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     const float new_max = fmaxf(smax, ptx::max3(fmaxf(m0, m1), m2, m3));
                     // Rescale by the difference of the two ROUNDED offsets: exactly 2^0 while the maximum
                     // stands, so no rounding residue compounds over the chunks of a long row.
-                    const float mb_new = new_max * c2;
+                    const float mb_new = fmaxf(new_max * c2, -3.0e38f);  // finite also while every column so far is masked
                     l *= ptx::ex2_approx(mb - mb_new);
                     mb = mb_new;
                     smax = new_max;

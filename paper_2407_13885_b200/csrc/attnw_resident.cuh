@@ -331,7 +331,7 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         bool ok = true;
 
         // sweep-1 state of the row block being accumulated
-        float smax = -3.0e38f, mb = smax * c2, l = 0.0f;
+        float smax = -3.0e38f, mb = -3.0e38f, l = 0.0f;
         float mb_slot[kSlots];  // the offset each slot's exponentials are relative to
 
         // Sweep 1 of one slot: local maximum, exponentials written back over the scores, local sum.
@@ -361,8 +361,8 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             m0 = ptx::max3(m0, s[28], s[29]);
             m1 = ptx::max3(m1, s[30], s[31]);
             const float new_max = fmaxf(smax, ptx::max3(fmaxf(m0, m1), m2, m3));
-            const float mb_new = new_max * c2;
-            l *= ptx::ex2_approx(mb - mb_new);  // exactly 1 while the maximum stands
+            const float mb_new = fmaxf(new_max * c2, -3.0e38f);  // finite also while every column so far is masked
+            l *= ptx::ex2_approx(mb - mb_new);                   // exactly 1 while the maximum stands
             mb = mb_new;
             smax = new_max;
             l += ragged ? exp2_chunk_inplace<kPoly, true>(s, c2c2, -mb, valid)
@@ -446,7 +446,7 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             for (int t = 0; t < kSlots; ++t) f_slot[t] = ptx::ex2_approx(mb_slot[t] - m_row) * inv_l;
             // reset the sweep-1 state for the next row block
             smax = -3.0e38f;
-            mb = smax * c2;
+            mb = -3.0e38f;
             l = 0.0f;
 
 #pragma unroll

@@ -156,6 +156,16 @@ def test_zero_scale_and_zero_queries_uniform(attnw):
     assert float((P - 1.0 / 200).abs().max()) <= 1e-7
 
 
+@pytest.mark.parametrize("variant", ["two_pass", "resident"])
+@pytest.mark.parametrize("N", [8, 72, 200])
+def test_large_scale_with_masked_columns(attnw, N, variant):
+    # scale * log2(e) > 1: the offset of a thread whose first columns are all beyond N must stay finite
+    q, k = small_fused_inputs(1, 2, N, 64, stream=77 + N)
+    P = run_fused(attnw, q, k, 2.0, torch.bfloat16, variant=variant)
+    assert bool(torch.isfinite(P.float()).all())
+    assert_close_to_oracle(P, oracle.attnw(q, k, 2.0), f"scale 2 N{N} {variant}")
+
+
 def test_key_permutation_permutes_columns(attnw):
     q, k = small_fused_inputs(1, 1, 512, 128, stream=9)
     perm = np.random.default_rng(5).permutation(512)
