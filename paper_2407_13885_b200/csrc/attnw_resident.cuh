@@ -45,6 +45,7 @@ enum : uint32_t {  // wait sites of this kernel (low byte of the status word)
     kSiteResExchange = 23,
     kSiteResStageFree = 24,
     kSiteResStageFilled = 25,
+    kSiteResStat = 26,
 };
 
 
@@ -64,8 +65,9 @@ struct ResidentSmem {
     static constexpr int kOutOff = kQOff + kTileBytes;                // staging boxes
     static constexpr int kPartOff = kOutOff + kStageBoxes * kBoxBytes;  // float2 part[4 column quarters][128 rows]
     static constexpr int kXchgOff = kPartOff + 4 * kTile * 8;         // float2 xchg[2 parities][8 CTAs][128 rows]
-    static constexpr int kBarOff = kXchgOff + 2 * kMaxClusterCtas * kTile * 8;
-    static constexpr int kBytes = kBarOff + 256;
+    static constexpr int kStatOff = kXchgOff + 2 * kMaxClusterCtas * kTile * 8;  // float2 stat[128 rows]: (M, 1/L)
+    static constexpr int kBarOff = kStatOff + kTile * 8;
+    static constexpr int kBytes = kBarOff + 512;
     static constexpr int kDynamicBytes = kBytes + 1024;
 };
 
@@ -74,12 +76,13 @@ struct ResidentBarriers {
     uint64_t s_full[kSlots], slot_free[kSlots];
     uint64_t part_full;
     uint64_t x_full[2];
+    uint64_t stat_full[4];
     uint64_t out_free[kStageBoxes], out_filled[kStageBoxes];
     uint32_t tmem_base;
     uint32_t abort_flag;
     uint32_t prior_failure;
 };
-static_assert(sizeof(ResidentBarriers) <= 256, "barrier block must fit its slot");
+static_assert(sizeof(ResidentBarriers) <= 512, "barrier block must fit its slot");
 
 // e_j = 2^(c2 * s_j + neg_offset) for one 32-column chunk, written over s; returns sum_j e_j.
 template <int POLY_PAIRS, bool RAGGED>
@@ -152,6 +155,7 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         ptx::mbar_init(&bars->part_full, kSoftmaxWarps);
         ptx::mbar_init(&bars->x_full[0], 1);
         ptx::mbar_init(&bars->x_full[1], 1);
+        for (int q = 0; q < 4; ++q) ptx::mbar_init(&bars->stat_full[q], 1);
         for (int b = 0; b < kStageBoxes; ++b) {
             ptx::mbar_init(&bars->out_free[b], 1);
             ptx::mbar_init(&bars->out_filled[b], 8);  // one arrival per Softmax warp of the column half
@@ -324,6 +328,7 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         float2* part = reinterpret_cast<float2*>(smem + L::kPartOff);
         const float2* xchg = reinterpret_cast<const float2*>(smem + L::kXchgOff);
         const uint32_t xchg_addr = ptx::smem_u32(smem + L::kXchgOff);
+        float2* stat = reinterpret_cast<float2*>(smem + L::kStatOff);
         const uint32_t out_base = ptx::smem_u32(smem + L::kOutOff);
         const uint32_t sw = static_cast<uint32_t>(row & 7);
         const bool stamp = warp == 0 && lane == 0;
@@ -425,22 +430,37 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             g += n_clusters;
             const bool have_next = g < total_items;
             // ---- global statistics of the current row block ----
+            // One thread per row (the warps of column quarter 0) reduces the cluster's pairs; the other three warps
+            // of the same TMEM lane quarter read (M, 1/L) from shared memory.  (The next write of stat[] follows
+            // this CTA's next post, which needs every warp to have passed this read.)
             const uint32_t par = item_n & 1u;
-            ok = __all_sync(0xffffffffu, fused_wait(&bars->x_full[par], (item_n >> 1) & 1u, abort_flag, kSiteResExchange));
-            if (!ok) break;
-            if (stamp) ATTNW_STAMP(4, item_n);
-            // all eight exchange slots are read at once (independent loads); slots beyond the cluster are ignored
-            float2 pc[kMaxClusterCtas];
+            float m_row, inv_l;
+            if (cq == 0) {
+                ok = __all_sync(0xffffffffu, fused_wait(&bars->x_full[par], (item_n >> 1) & 1u, abort_flag, kSiteResExchange));
+                if (!ok) break;
+                if (stamp) ATTNW_STAMP(4, item_n);
+                // all eight exchange slots are read at once (independent loads); slots beyond the cluster are ignored
+                float2 pc[kMaxClusterCtas];
 #pragma unroll
-            for (int c = 0; c < kMaxClusterCtas; ++c) pc[c] = xchg[(par * kMaxClusterCtas + c) * kTile + row];
-            float m_row = pc[0].x;
+                for (int c = 0; c < kMaxClusterCtas; ++c) pc[c] = xchg[(par * kMaxClusterCtas + c) * kTile + row];
+                m_row = pc[0].x;
 #pragma unroll
-            for (int c = 1; c < kMaxClusterCtas; ++c) m_row = (c < cluster_ctas) ? fmaxf(m_row, pc[c].x) : m_row;
-            float l_row = 0.0f;
+                for (int c = 1; c < kMaxClusterCtas; ++c) m_row = (c < cluster_ctas) ? fmaxf(m_row, pc[c].x) : m_row;
+                float l_row = 0.0f;
 #pragma unroll
-            for (int c = 0; c < kMaxClusterCtas; ++c)
-                l_row += (c < cluster_ctas) ? pc[c].y * ptx::ex2_approx(pc[c].x - m_row) : 0.0f;
-            const float inv_l = 1.0f / l_row;
+                for (int c = 0; c < kMaxClusterCtas; ++c)
+                    l_row += (c < cluster_ctas) ? pc[c].y * ptx::ex2_approx(pc[c].x - m_row) : 0.0f;
+                inv_l = 1.0f / l_row;
+                stat[row] = make_float2(m_row, inv_l);
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&bars->stat_full[quarter]);
+            } else {
+                ok = __all_sync(0xffffffffu, fused_wait(&bars->stat_full[quarter], item_n & 1u, abort_flag, kSiteResStat));
+                if (!ok) break;
+                const float2 ml = stat[row];
+                m_row = ml.x;
+                inv_l = ml.y;
+            }
             float f_slot[kSlots];
 #pragma unroll
             for (int t = 0; t < kSlots; ++t) f_slot[t] = ptx::ex2_approx(mb_slot[t] - m_row) * inv_l;
