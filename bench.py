@@ -37,7 +37,10 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
 # summarised under profiles/; None until a capture exists for that kernel.
-NCU_TRAFFIC_BYTES = {"c3": 8 * (33.64e6 + 476.31e6), "c3_two_pass": 8 * (33.97e6 + 477.69e6),
+# (c3, default variant: the split launch gives 107 of 128 heads to the resident kernel and 21 to the two-pass
+# kernel; each kernel's capture covers 16 heads, so the launch's traffic is the head-weighted sum.)
+NCU_TRAFFIC_BYTES = {"c3": (107 * (33.64e6 + 476.31e6) + 21 * (33.97e6 + 477.69e6)) / 16,
+                     "c3_resident": 8 * (33.64e6 + 476.31e6), "c3_two_pass": 8 * (33.97e6 + 477.69e6),
                      "c4": 4 * (268.45e6 + 98.18e6)}
 
 
@@ -379,7 +382,7 @@ def run_ours(args):
     t_flop = w.flops / (peaks["bf16_tflops"] * 1e12)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"],
-                "traffic": NCU_TRAFFIC_BYTES.get(w.name + ("_two_pass" if args.variant == "two_pass" else "")),
+                "traffic": NCU_TRAFFIC_BYTES.get(w.name + {"two_pass": "_two_pass", "resident": "_resident"}.get(args.variant, "")),
                 "peak_source": f"of {peaks['source']}",
                 "algorithmic_bytes_per_launch": bytes_alg,
                 "roofline_time_us": 1e6 * max(t_hbm, t_flop), "kernel_time_us": 1e6 * kernel_s,
