@@ -59,9 +59,9 @@ int attnw_fused_f32(const void* Q, const void* K, void* P, int B, int H, int N, 
 
 /*
  * Which kernel attnw_fused uses (process-wide; the results are the same within the stated tolerances):
- *   0  choose by shape (default): the SRAM-resident kernel when P is bfloat16, N <= 4096 and every
- *      cluster has at least 32 row blocks of 128 queries to walk; the two-pass kernel otherwise
- *      (and always for attnw_fused_f32).  Clusters of 8 cannot occupy every SM, so such a call is
+ *   0  choose by shape (default): the SRAM-resident kernel when P is bfloat16 and N <= 4096; the
+ *      two-pass kernel otherwise (and always for attnw_fused_f32).  Clusters cannot occupy every SM
+ *      (clusters of 8: 120 of 148), so a large call is
  *      split: most heads go to the resident kernel on `stream`, the rest to the two-pass kernel on a
  *      per-device side stream that forks from and joins `stream` with events (first use creates the
  *      side stream and two events); work enqueued on `stream` afterwards sees the whole result.

@@ -239,12 +239,11 @@ int fused_entry(const void* Q, const void* K, void* P, int B, int H, int N, int 
     const int variant = g_fused_variant.load(std::memory_order_relaxed);
     const bool resident_fits = sizeof(OutT) == 2 && N <= kResidentMaxN;
     if (variant == 2 && !resident_fits) return ATTNW_ERR_UNSUPPORTED;
-    // Choice by shape: the resident kernel wins once every cluster has a long list of row blocks to walk
-    // (measured: 1.46 vs 1.52 ms at B*H = 128, N = 4096, d = 128); with few row blocks per cluster its
-    // set-up and its exchange latency are not amortised (0.057 vs 0.049 ms at B*H = 12, N = 2048, d = 64).
-    const long long row_blocks = static_cast<long long>(B) * H * ((N + kTile - 1) / kTile);
-    const long long clusters_at_most = dev->sm_count / ((N + kSlab - 1) / kSlab);
-    const bool resident_pays = row_blocks >= 32 * clusters_at_most;
+    // Choice by shape: the resident kernel whenever it can serve the call.  It spreads one 128-row block over the
+    // C SMs of a cluster, so it also fills the device when B*H is small (B*H = 1, N = 4096, d = 128: 25 us
+    // against 96 us; B*H = 12, N = 2048, d = 64: 37 against 51 us); between B*H = 8 and 16 at N = 4096 the
+    // two kernels are within 2 % of each other, above that the resident kernel leads again.
+    const bool resident_pays = true;
     if (resident_fits && (variant == 2 || (variant == 0 && resident_pays))) {
         if constexpr (sizeof(OutT) == 2) {
             // Clusters of 8 cannot occupy every SM (15 x 8 = 120 of 148 on B200).  When the call is chosen by

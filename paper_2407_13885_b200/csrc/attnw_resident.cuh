@@ -426,7 +426,6 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             post_partials(item_n);
         }
         while (have && ok) {
-            const int cur_bh = g / T, cur_rb = g % T;
             g += n_clusters;
             const bool have_next = g < total_items;
             // ---- global statistics of the current row block ----

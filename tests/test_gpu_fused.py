@@ -62,6 +62,17 @@ def test_resident_variant_matches_oracle(attnw, B, H, N, d):
     assert_close_to_oracle(P, oracle.attnw(q, k, scale), f"resident B{B} H{H} N{N} d{d}")
 
 
+def test_default_choice_splits_a_call_over_both_kernels(attnw):
+    # B*H = 32, N = 2048: 33 clusters of 4 leave 16 SMs idle and walk 16 rounds of row blocks, so the default
+    # choice gives two heads to the two-pass kernel on a side stream; the whole of P must be there afterwards
+    q, k = small_fused_inputs(4, 8, 2048, 64, stream=99)
+    scale = float(np.float32(0.125))
+    attnw.launch_count(reset=True)
+    P = run_fused(attnw, q, k, scale, torch.bfloat16, variant="auto")
+    assert attnw.launch_count() == 2
+    assert_close_to_oracle(P, oracle.attnw(q, k, scale), "split launch B4 H8 N2048 d64")
+
+
 def test_resident_variant_large_logits_and_limits(attnw):
     q, k = small_fused_inputs(1, 2, 2048, 128, sigma=4.0, stream=56)
     scale = float(np.float32(1.0 / math.sqrt(128.0)))
