@@ -32,6 +32,7 @@ struct DeviceInfo {
     bool ready = false;
     int cc_major = 0;
     int sm_count = 0;
+    int fused_pairs[2][2] = {};  // [d == 128][float32 P]: co-resident two-CTA clusters of the two-pass kernel, 0 = not asked yet
     int resident_clusters[2][kMaxClusterCtas + 1] = {};  // [d == 128][cluster size]: co-resident clusters, 0 = not asked yet
     // fork/join objects for launches that split a call over two kernels (created on first use)
     cudaStream_t side_stream = nullptr;
@@ -123,7 +124,7 @@ int validate_fused(const void* Q, const void* K, const void* P, int B, int H, in
 
 template <int D, typename OutT>
 int launch_fused(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH, int N, float scale,
-                 cudaStream_t stream) {
+                 cudaStream_t stream, bool allow_key_split = true) {
     using L = FusedSmem<D>;
     auto kernel = attnw_fused_kernel<D, OutT>;
     CUtensorMap tm_q, tm_k, tm_p;
@@ -141,11 +142,62 @@ int launch_fused(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH,
         (void)cudaGetLastError();
         return ATTNW_ERR_CUDA;
     }
-    (void)dev;
     const int row_blocks = (N + kRowsPerCta - 1) / kRowsPerCta;
     const float scale_log2e = static_cast<float>(static_cast<double>(scale) * 1.4426950408889634074);
-    kernel<<<static_cast<unsigned>(BH * row_blocks), kFusedThreads, L::kDynamicBytes, stream>>>(tm_q, tm_k, tm_p, N,
-                                                                                                 row_blocks, scale_log2e);
+    const long long ctas = static_cast<long long>(BH) * row_blocks;
+    // Two CTAs per 256-row block (each walks half of the key tiles; see the kernel) when that fills the device
+    // better: CTAs of half the length in waves of `pairs` clusters against whole CTAs in waves of `sm_count`
+    // (N = 16384, B*H = 8: 512 CTAs = 4 waves of 148 become 7 half-length waves of 74 pairs; a call with fewer
+    // CTAs than SMs simply finishes in half the time).
+    int key_split = 1;
+    if (allow_key_split && ((N + kTile - 1) / kTile) % 2 == 0 && 2 * ctas <= INT_MAX) {
+        int& pairs = dev->fused_pairs[D == 128 ? 1 : 0][sizeof(OutT) == 2 ? 0 : 1];
+        if (pairs == 0) {
+            cudaLaunchAttribute a[1];
+            a[0].id = cudaLaunchAttributeClusterDimension;
+            a[0].val.clusterDim.x = 2;
+            a[0].val.clusterDim.y = 1;
+            a[0].val.clusterDim.z = 1;
+            cudaLaunchConfig_t c = {};
+            c.blockDim = dim3(kFusedThreads, 1, 1);
+            c.gridDim = dim3(static_cast<unsigned>(2 * dev->sm_count), 1, 1);
+            c.dynamicSmemBytes = L::kDynamicBytes;
+            c.attrs = a;
+            c.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, kernel, &c) != cudaSuccess || n < 1) {
+                (void)cudaGetLastError();
+                n = -1;
+            }
+            pairs = n;
+        }
+        if (pairs > 0) {
+            const long long whole_waves = (ctas + dev->sm_count - 1) / dev->sm_count;
+            const long long half_waves = (ctas + pairs - 1) / pairs;
+            if (half_waves * 51 < whole_waves * 100) key_split = 2;  // 2 % for the exchange
+        }
+    }
+    if (key_split == 1) {
+        kernel<<<static_cast<unsigned>(ctas), kFusedThreads, L::kDynamicBytes, stream>>>(tm_q, tm_k, tm_p, N, row_blocks,
+                                                                                         scale_log2e, 1);
+    } else {
+        cudaLaunchAttribute a[1];
+        a[0].id = cudaLaunchAttributeClusterDimension;
+        a[0].val.clusterDim.x = 2;
+        a[0].val.clusterDim.y = 1;
+        a[0].val.clusterDim.z = 1;
+        cudaLaunchConfig_t c = {};
+        c.blockDim = dim3(kFusedThreads, 1, 1);
+        c.gridDim = dim3(static_cast<unsigned>(2 * ctas), 1, 1);
+        c.dynamicSmemBytes = L::kDynamicBytes;
+        c.stream = stream;
+        c.attrs = a;
+        c.numAttrs = 1;
+        if (cudaLaunchKernelEx(&c, kernel, tm_q, tm_k, tm_p, N, row_blocks, scale_log2e, 2) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return ATTNW_ERR_CUDA;
+        }
+    }
     if (cudaGetLastError() != cudaSuccess) return ATTNW_ERR_CUDA;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return ATTNW_OK;
@@ -294,8 +346,8 @@ int fused_entry(const void* Q, const void* K, void* P, int B, int H, int N, int 
                                : launch_resident<128>(dev, Q, K, P, bh_res, N, scale, s);
                 if (rc != ATTNW_OK) return rc;
                 if (cudaStreamWaitEvent(dev->side_stream, dev->fork_event, 0) != cudaSuccess) return ATTNW_ERR_CUDA;
-                rc = (d == 64) ? launch_fused<64, OutT>(dev, q2, k2, p2, bh_two_pass, N, scale, dev->side_stream)
-                               : launch_fused<128, OutT>(dev, q2, k2, p2, bh_two_pass, N, scale, dev->side_stream);
+                rc = (d == 64) ? launch_fused<64, OutT>(dev, q2, k2, p2, bh_two_pass, N, scale, dev->side_stream, false)
+                               : launch_fused<128, OutT>(dev, q2, k2, p2, bh_two_pass, N, scale, dev->side_stream, false);
                 if (cudaEventRecord(dev->join_event, dev->side_stream) != cudaSuccess ||
                     cudaStreamWaitEvent(s, dev->join_event, 0) != cudaSuccess)
                     return ATTNW_ERR_CUDA;

@@ -87,6 +87,7 @@ enum : uint32_t {  // which wait gave up (low byte of the status word)
     kSiteSoftmaxNorm = 6,
     kSiteStageFree = 7,
     kSiteStageFilled = 8,
+    kSitePair = 9,
 };
 
 template <int D>
@@ -111,6 +112,7 @@ struct FusedBarriers {
     uint64_t s_empty[2][2];
     uint64_t out_free[4];    // [query tile * 2 + column half]: the staging buffer has been read by its store
     uint64_t out_filled[4];  // ... has been filled by the three warps that do not issue the store
+    uint64_t pair_full;      // two CTAs per row block: the partner's statistics have arrived
     uint32_t tmem_base;
     uint32_t abort_flag;
     uint32_t prior_failure;
@@ -208,7 +210,8 @@ __device__ __forceinline__ float sum_exp2_chunk(const float (&s)[kChunk], uint64
 template <int D, typename OutT>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                   const __grid_constant__ CUtensorMap tm_p, int N, int row_blocks_per_head, float scale_log2e) {
+                   const __grid_constant__ CUtensorMap tm_p, int N, int row_blocks_per_head, float scale_log2e,
+                   int key_split) {
     using L = FusedSmem<D>;
     constexpr bool kBf16Out = sizeof(OutT) == 2;
     constexpr int kPolyStats = kBf16Out ? ATTNW_POLY_PAIRS_STATS : 0;
@@ -227,13 +230,26 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
 #endif
     if (threadIdx.x == 0) bars->prior_failure = *reinterpret_cast<volatile unsigned int*>(&g_attnw_status);
     __syncthreads();
-    if (bars->prior_failure != 0u) return;  // an earlier CTA gave up: do not queue more waits behind it
+    if (bars->prior_failure != 0u) {  // an earlier CTA gave up: do not queue more waits behind it
+        if (key_split > 1) {          // (the partner CTA still passes the one cluster barrier of the set-up)
+            ptx::cluster_arrive_release();
+            ptx::cluster_wait_acquire();
+        }
+        return;
+    }
 
+    // key_split = 1: one CTA per 256 rows walks all key tiles.  key_split = 2: a cluster of two CTAs shares the 256
+    // rows; each walks half of the key tiles in both passes and the two exchange their rows' (offset, sum) between
+    // the passes through distributed shared memory - the exchange of local maxima and sums of Section VII, here only
+    // to fill the device when the CTAs do not divide evenly over the SMs or are fewer than the SMs.
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int bh = blockIdx.x / row_blocks_per_head;
-    const int row0 = (blockIdx.x % row_blocks_per_head) * kRowsPerCta;
-    const int T = (N + kTile - 1) / kTile;  // key tiles per pass
+    const uint32_t pair_rank = key_split > 1 ? ptx::cluster_ctarank() : 0u;
+    const int unit = static_cast<int>(blockIdx.x) / key_split;
+    const int bh = unit / row_blocks_per_head;
+    const int row0 = (unit % row_blocks_per_head) * kRowsPerCta;
+    const int T = ((N + kTile - 1) / kTile) / key_split;  // key tiles of this CTA per pass
+    const int kt0 = static_cast<int>(pair_rank) * T;      // its first key tile
     const int total_iters = 2 * T;
     const bool tile_active[2] = {row0 < N, row0 + kTile < N};
 
@@ -253,8 +269,11 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             ptx::mbar_init(&bars->out_free[g], 1);
             ptx::mbar_init(&bars->out_filled[g], 3);
         }
+        ptx::mbar_init(&bars->pair_full, 1);
         bars->abort_flag = 0;
         ptx::mbar_fence_init();
+        if (key_split > 1)  // the partner's 512 (256) threads each send 8 bytes for their row
+            ptx::mbar_expect_tx(&bars->pair_full, ((tile_active[0] ? 1u : 0u) + (tile_active[1] ? 1u : 0u)) * 2048u);
     }
     if (warp == kProducerWarp && lane == 0) {
         ptx::prefetch_tensormap(&tm_q);
@@ -267,6 +286,10 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (key_split > 1) {  // the partner writes into this CTA's shared memory: not before its barrier exists
+        ptx::cluster_arrive_release();
+        ptx::cluster_wait_acquire();
+    }
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
 
@@ -295,7 +318,7 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 }
 #endif
                 ptx::mbar_expect_tx(&bars->k_full[s], static_cast<uint32_t>(L::kTileBytes));
-                const int kt = it < T ? it : it - T;
+                const int kt = kt0 + (it < T ? it : it - T);
                 for (int a = 0; a < L::kAtoms; ++a)
                     ptx::tma_load_3d(smem + L::kKOff + s * L::kTileBytes + a * L::kAtomBytes, &tm_k, &bars->k_full[s],
                                      a * 64, kt * kTile, bh, keep);
@@ -399,7 +422,7 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         if (lane == 0) ptx::mbar_arrive(&bars->s_empty[q][buf]);
                         if (stamp) ATTNW_STAMP(8 + q * 4, it);
                     }
-                    const int valid = N - it * kTile - half * kHalf - c * kChunk;  // columns of this chunk that exist
+                    const int valid = N - (kt0 + it) * kTile - half * kHalf - c * kChunk;  // columns of this chunk that exist
                     const bool ragged = valid < kChunk;
                     if (ragged) {
 #pragma unroll
@@ -444,6 +467,22 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 l = l * ptx::ex2_approx(mb - mb_row) + other.y * ptx::ex2_approx(other.x - mb_row);
                 mb = mb_row;
             }
+            // ---- two CTAs per row block: add the partner's half of the keys ----
+            if (key_split > 1) {
+                // every thread sends its row's pair to the thread of the same warp and lane in the partner CTA, into
+                // bytes 256.. of that warp's staging buffer (idle until the normalise pass; bytes 0..255 served the
+                // merge above), and waits - bounded - for the partner's
+                const uint32_t inbox = ptx::smem_u32(smem + L::kOutOff + warp * kStageBoxBytes + 256 + lane * 8);
+                ptx::st_async_b64(ptx::map_to_cta(inbox, pair_rank ^ 1u), ptx::pack2(mb, l),
+                                  ptx::map_to_cta(ptx::smem_u32(&bars->pair_full), pair_rank ^ 1u));
+                ok = __all_sync(0xffffffffu, ok && fused_wait(&bars->pair_full, 0, abort_flag, kSitePair));
+                if (ok) {
+                    const float2 other = *reinterpret_cast<const float2*>(smem + L::kOutOff + warp * kStageBoxBytes + 256 + lane * 8);
+                    const float mb_row = fmaxf(mb, other.x);
+                    l = l * ptx::ex2_approx(mb - mb_row) + other.y * ptx::ex2_approx(other.x - mb_row);
+                    mb = mb_row;
+                }
+            }
 
             // ---- normalise pass: p = 2^(c2*s - (mb + log2 l)), stored once ----
             // bf16 output: 1/l is folded into the exponent (one FFMA + one exponential per element); the
@@ -466,7 +505,7 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             const uint64_t stream_out = ptx::policy_evict_first();
             const uint64_t nshift2 = ptx::pack2(-shift, -shift);
             for (int it = T; ok && it < total_iters; ++it) {
-                const int kt = it - T;
+                const int kt = kt0 + it - T;
                 const int buf = it & 1;
                 if (stamp) ATTNW_STAMP(6 + q * 4, it);
                 ok = fused_wait(&bars->s_full[q][buf], static_cast<uint32_t>(it >> 1) & 1u, abort_flag,
