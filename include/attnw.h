@@ -66,9 +66,10 @@ int attnw_fused_f32(const void* Q, const void* K, void* P, int B, int H, int N, 
  *      per-device side stream that forks from and joins `stream` with events (first use creates the
  *      side stream and two events); work enqueued on `stream` afterwards sees the whole result.
  *   1  two-pass kernel: statistics pass + normalise pass that recomputes the score tiles; any N
- *   2  SRAM-resident kernel: a cluster of ceil(N/512) CTAs keeps a 128-row block of scores in tensor
+ *   2  SRAM-resident kernel: a cluster of ceil(N/512) <= 16 CTAs keeps a 128-row block of scores in tensor
  *      memory and exchanges local row maxima and sums across CTAs, as the fused kernel of Section VII
- *      does across Tensix cores; a call it cannot serve then returns ATTNW_ERR_UNSUPPORTED
+ *      does across Tensix cores; serves bfloat16 P and N <= 8192, any other call then returns
+ *      ATTNW_ERR_UNSUPPORTED
  * Returns ATTNW_ERR_BAD_SHAPE for any other value.
  */
 int attnw_set_fused_variant(int variant);

@@ -204,13 +204,14 @@ int launch_fused(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH,
 }
 
 // How many clusters of `cluster_ctas` CTAs of the resident kernel the device can hold at once (cached).
-template <int D>
-int resident_max_clusters(DeviceInfo* dev, int cluster_ctas) {
+template <int D, int CMAX>
+int resident_max_clusters_impl(DeviceInfo* dev, int cluster_ctas) {
     int& cached = dev->resident_clusters[D == 128 ? 1 : 0][cluster_ctas];
     if (cached != 0) return cached;
-    using L = ResidentSmem<D>;
-    auto kernel = attnw_resident_kernel<D>;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess) {
+    using L = ResidentSmem<D, CMAX>;
+    auto kernel = attnw_resident_kernel<D, CMAX>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess ||
+        (CMAX > 8 && cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)) {
         (void)cudaGetLastError();
         return cached = -1;
     }
@@ -233,19 +234,26 @@ int resident_max_clusters(DeviceInfo* dev, int cluster_ctas) {
     return cached = n;
 }
 
+template <int D>
+int resident_max_clusters(DeviceInfo* dev, int cluster_ctas) {
+    return cluster_ctas <= 8 ? resident_max_clusters_impl<D, 8>(dev, cluster_ctas)
+                             : resident_max_clusters_impl<D, 16>(dev, cluster_ctas);
+}
+
 // SRAM-resident single-pass kernel: one cluster of ceil(N / 512) CTAs per 128-row block, persistent over
 // a list of row blocks.  Returns ATTNW_ERR_UNSUPPORTED when the device cannot co-schedule such a cluster.
-template <int D>
-int launch_resident(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH, int N, float scale,
-                    cudaStream_t stream) {
-    using L = ResidentSmem<D>;
-    auto kernel = attnw_resident_kernel<D>;
+template <int D, int CMAX>
+int launch_resident_impl(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH, int N, float scale,
+                         cudaStream_t stream) {
+    using L = ResidentSmem<D, CMAX>;
+    auto kernel = attnw_resident_kernel<D, CMAX>;
     CUtensorMap tm_q, tm_k, tm_p;
     int rc = encode_3d(&tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Q, D, N, BH, 64, kTile);
     if (rc == ATTNW_OK) rc = encode_3d(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, K, D, N, BH, 64, kTile);
     if (rc == ATTNW_OK) rc = encode_3d(&tm_p, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, P, N, N, BH, 64, kTile);
     if (rc != ATTNW_OK) return rc;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess ||
+        (CMAX > 8 && cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)) {
         (void)cudaGetLastError();
         return ATTNW_ERR_CUDA;
     }
@@ -278,6 +286,13 @@ int launch_resident(DeviceInfo* dev, const void* Q, const void* K, void* P, int 
     return ATTNW_OK;
 }
 
+template <int D>
+int launch_resident(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH, int N, float scale,
+                    cudaStream_t stream) {
+    return (N + kSlab - 1) / kSlab <= 8 ? launch_resident_impl<D, 8>(dev, Q, K, P, BH, N, scale, stream)
+                                        : launch_resident_impl<D, 16>(dev, Q, K, P, BH, N, scale, stream);
+}
+
 template <typename OutT>
 int fused_entry(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream) {
     int rc = validate_fused(Q, K, P, B, H, N, d, scale, sizeof(OutT));
@@ -295,7 +310,10 @@ int fused_entry(const void* Q, const void* K, void* P, int B, int H, int N, int 
     // C SMs of a cluster, so it also fills the device when B*H is small (B*H = 1, N = 4096, d = 128: 25 us
     // against 96 us; B*H = 12, N = 2048, d = 64: 37 against 51 us); between B*H = 8 and 16 at N = 4096 the
     // two kernels are within 2 % of each other, above that the resident kernel leads again.
-    const bool resident_pays = true;
+    // Clusters of more than 8 CTAs (N > 4096) fit only 7 times (112 SMs): there the two-pass kernel with two CTAs per
+    // row block is ahead except for a single head (B*H = 4, N = 8192: 188 against 221 us), so the choice by shape
+    // stops at N = 4096; variant 2 serves N <= 8192 on request.
+    const bool resident_pays = N <= 8 * kSlab;
     if (resident_fits && (variant == 2 || (variant == 0 && resident_pays))) {
         if constexpr (sizeof(OutT) == 2) {
             // Clusters of 8 cannot occupy every SM (15 x 8 = 120 of 148 on B200).  When the call is chosen by

@@ -3,7 +3,7 @@
 //
 // The paper lays the whole score matrix out over a grid of cores, keeps every core's block of scores
 // in its SRAM, computes LOCAL row maxima and row sums per core and exchanges them along a grid row
-// to obtain the GLOBAL ones before normalising (Section VII; Eq. 1).  Here a cluster of C <= 8 CTAs
+// to obtain the GLOBAL ones before normalising (Section VII; Eq. 1).  Here a cluster of C <= 16 CTAs
 // owns a 128-row block of one head; CTA r keeps the 128 x 512 slab of scores for keys
 // [512 r, 512 r + 512) in its tensor memory (all 512 TMEM columns), so the tensor cores and the
 // exponentials run ONCE per element (the two-pass kernel runs both twice):
@@ -16,7 +16,7 @@
 //            issuer, which already computes the next row block's scores into it.
 // A cluster walks whole units of work (a head, or a range of its row blocks), so the CTA's key slab is
 // loaded into shared memory once per unit and only the 32 KB query tiles stream.
-// Valid for N <= 8 * 512 = 4096 keys and bf16 output; anything else takes the two-pass kernel.
+// Valid for N <= 16 * 512 = 8192 keys and bf16 output; anything else takes the two-pass kernel.
 #pragma once
 #include "attnw_fused.cuh"
 
@@ -26,7 +26,7 @@ constexpr int kSlab = 512;                 // key columns per CTA: one full tens
 constexpr int kSlots = kSlab / kTile;      // accumulator slots of 128 columns
 constexpr int kResidentThreads = 608;      // 16 Softmax warps + TMA producer + MMA issuer + store issuer
 constexpr int kStoreWarp = 18;
-constexpr int kMaxClusterCtas = 8;         // portable cluster size limit
+constexpr int kMaxClusterCtas = 16;        // largest cluster; sizes above 8 are non-portable and the launch opts in
 constexpr int kResidentMaxN = kSlab * kMaxClusterCtas;
 constexpr int kBoxBytes = kTile * 128;     // one staged store box: 128 rows x 128 bytes
 
@@ -52,11 +52,14 @@ enum : uint32_t {  // wait sites of this kernel (low byte of the status word)
 constexpr int kKStages = 2;        // key sub-tiles in flight in shared memory
 constexpr int kS1Lag = 1;          // sweep 1 of the next row block trails sweep 2 of the current one by this many slots
 constexpr int kStoreLag = 3;       // stores allowed to be still reading shared memory when the next one is issued
-constexpr int kStageBoxes = 6;     // staged store boxes: three per column half, so that about 100 KB of
+constexpr int kStageBoxesMax = 6;  // staged store boxes: three per column half, so that about 100 KB of
                                    // stores can be in flight (the write path needs that much to stay busy)
 
-template <int D>
+// CMAX = 8 or 16: the largest cluster an instantiation serves.  It sizes the exchange area; with 16 one staging box
+// makes room for it.  (The instantiation for CMAX = 8 is the one the headline workload runs.)
+template <int D, int CMAX>
 struct ResidentSmem {
+    static constexpr int kStageBoxes = (CMAX <= 8) ? 6 : 5;
     static constexpr int kAtoms = D / 64;
     static constexpr int kAtomBytes = kTile * 128;
     static constexpr int kTileBytes = kAtoms * kAtomBytes;
@@ -65,11 +68,14 @@ struct ResidentSmem {
     static constexpr int kOutOff = kQOff + kTileBytes;                // staging boxes
     static constexpr int kPartOff = kOutOff + kStageBoxes * kBoxBytes;  // float2 part[4 column quarters][128 rows]
     static constexpr int kXchgOff = kPartOff + 4 * kTile * 8;         // float2 xchg[2 parities][8 CTAs][128 rows]
-    static constexpr int kStatOff = kXchgOff + 2 * kMaxClusterCtas * kTile * 8;  // float2 stat[128 rows]: (M, 1/L)
+    static constexpr int kStatOff = kXchgOff + 2 * CMAX * kTile * 8;  // float2 stat[128 rows]: (M, 1/L)
     static constexpr int kBarOff = kStatOff + kTile * 8;
     static constexpr int kBytes = kBarOff + 512;
     static constexpr int kDynamicBytes = kBytes + 1024;
 };
+
+static_assert(ResidentSmem<128, 8>::kDynamicBytes <= 227 * 1024 && ResidentSmem<128, 16>::kDynamicBytes <= 227 * 1024,
+              "shared memory budget");
 
 struct ResidentBarriers {
     uint64_t k_full[kKStages], k_empty[kKStages], q_full, q_empty;
@@ -77,7 +83,7 @@ struct ResidentBarriers {
     uint64_t part_full;
     uint64_t x_full[2];
     uint64_t stat_full[4];
-    uint64_t out_free[kStageBoxes], out_filled[kStageBoxes];
+    uint64_t out_free[kStageBoxesMax], out_filled[kStageBoxesMax];
     uint32_t tmem_base;
     uint32_t abort_flag;
     uint32_t prior_failure;
@@ -118,12 +124,13 @@ __device__ __forceinline__ float exp2_chunk_inplace(float (&s)[kChunk], uint64_t
 // Work list: item g = (head g / T, row block g % T); cluster c takes items c, c + G, c + 2G, ...  (neighbouring
 // clusters work on neighbouring row blocks of one head, so its keys stay hot in L2).  Every role of every CTA
 // of the cluster walks the same list.
-template <int D>
+template <int D, int CMAX>
 __global__ void __launch_bounds__(kResidentThreads, 1)
 attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                       const __grid_constant__ CUtensorMap tm_p, int N, int total_items, int cluster_ctas,
                       float scale_log2e) {
-    using L = ResidentSmem<D>;
+    using L = ResidentSmem<D, CMAX>;
+    constexpr int kStageBoxes = L::kStageBoxes;
     constexpr int kPoly = ATTNW_POLY_PAIRS_RESIDENT;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -402,7 +409,7 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 if (warp == 0 && lane == 0)  // arm this CTA's receive barrier for the whole cluster's rows
                     ptx::mbar_expect_tx(&bars->x_full[par], static_cast<uint32_t>(cluster_ctas * kTile * 8));
                 const uint64_t payload = ptx::pack2(mc, lc);
-                const uint32_t slot_addr = xchg_addr + ((par * kMaxClusterCtas + rank) * kTile + row) * 8u;
+                const uint32_t slot_addr = xchg_addr + ((par * CMAX + rank) * kTile + row) * 8u;
                 const uint32_t bar_addr = ptx::smem_u32(&bars->x_full[par]);
                 for (int dst = 0; dst < cluster_ctas; ++dst)
                     ptx::st_async_b64(ptx::map_to_cta(slot_addr, dst), payload, ptx::map_to_cta(bar_addr, dst));
@@ -439,15 +446,15 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 if (!ok) break;
                 if (stamp) ATTNW_STAMP(4, item_n);
                 // all eight exchange slots are read at once (independent loads); slots beyond the cluster are ignored
-                float2 pc[kMaxClusterCtas];
+                float2 pc[CMAX];
 #pragma unroll
-                for (int c = 0; c < kMaxClusterCtas; ++c) pc[c] = xchg[(par * kMaxClusterCtas + c) * kTile + row];
+                for (int c = 0; c < CMAX; ++c) pc[c] = xchg[(par * CMAX + c) * kTile + row];
                 m_row = pc[0].x;
 #pragma unroll
-                for (int c = 1; c < kMaxClusterCtas; ++c) m_row = (c < cluster_ctas) ? fmaxf(m_row, pc[c].x) : m_row;
+                for (int c = 1; c < CMAX; ++c) m_row = (c < cluster_ctas) ? fmaxf(m_row, pc[c].x) : m_row;
                 float l_row = 0.0f;
 #pragma unroll
-                for (int c = 0; c < kMaxClusterCtas; ++c)
+                for (int c = 0; c < CMAX; ++c)
                     l_row += (c < cluster_ctas) ? pc[c].y * ptx::ex2_approx(pc[c].x - m_row) : 0.0f;
                 inv_l = 1.0f / l_row;
                 stat[row] = make_float2(m_row, inv_l);

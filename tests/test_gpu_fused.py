@@ -48,10 +48,10 @@ def test_fused_matches_oracle(attnw, B, H, N, d, dtype):
     assert_close_to_oracle(P, oracle.attnw(q, k, scale), f"B{B} H{H} N{N} d{d}")
 
 
-# The SRAM-resident cluster kernel: cluster sizes 1..8, ragged slabs, a last CTA with one to four slots in use.
+# The SRAM-resident cluster kernel: cluster sizes 1..16, ragged slabs, a last CTA with one to four slots in use.
 RESIDENT_SHAPES = [(1, 1, 128, 64), (1, 1, 512, 128), (1, 2, 1024, 128), (1, 3, 384, 64), (2, 2, 2048, 64),
                    (1, 2, 4096, 128), (1, 1, 200, 128), (1, 1, 1160, 64), (1, 2, 2568, 128), (1, 1, 8, 64),
-                   (1, 1, 3080, 64), (3, 5, 640, 128)]
+                   (1, 1, 3080, 64), (3, 5, 640, 128), (1, 1, 4608, 64), (1, 1, 5000, 128), (1, 2, 8192, 64)]
 
 
 @pytest.mark.parametrize("B,H,N,d", RESIDENT_SHAPES)
@@ -85,7 +85,7 @@ def test_resident_variant_large_logits_and_limits(attnw):
     P = run_fused(attnw, q, kk, 0.3, torch.bfloat16, variant="resident")
     assert bool((P == 1.0 / 2048).all())
     # beyond its range, or for float32 output, the resident kernel refuses instead of silently switching
-    big = torch.zeros((1, 1, 4104, 64), dtype=torch.bfloat16, device="cuda")
+    big = torch.zeros((1, 1, 8200, 64), dtype=torch.bfloat16, device="cuda")
     attnw.set_fused_variant("resident")
     try:
         with pytest.raises(attnw.AttnwError) as e:
