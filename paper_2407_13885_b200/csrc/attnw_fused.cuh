@@ -231,7 +231,9 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     if (threadIdx.x == 0) bars->prior_failure = *reinterpret_cast<volatile unsigned int*>(&g_attnw_status);
     __syncthreads();
     if (bars->prior_failure != 0u) {  // an earlier CTA gave up: do not queue more waits behind it
-        if (key_split > 1) {          // (the partner CTA still passes the one cluster barrier of the set-up)
+        if (key_split > 1) {          // (the partner CTA still passes the cluster barriers of set-up and teardown)
+            ptx::cluster_arrive_release();
+            ptx::cluster_wait_acquire();
             ptx::cluster_arrive_release();
             ptx::cluster_wait_acquire();
         }
@@ -608,6 +610,10 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     // ---- teardown: every role falls through to here, also after a wait gave up ----
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (key_split > 1) {  // the partner may still be sending its statistics into this CTA's shared memory
+        ptx::cluster_arrive_release();
+        ptx::cluster_wait_acquire();
+    }
     if (warp == kMmaWarp) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
