@@ -39,8 +39,8 @@ FALLBACK_BF16_TFLOPS = 1590.0
 # summarised under profiles/; None until a capture exists for that kernel.
 # (c3, default variant: the split launch gives 107 of 128 heads to the resident kernel and 21 to the two-pass
 # kernel; each kernel's capture covers 16 heads, so the launch's traffic is the head-weighted sum.)
-NCU_TRAFFIC_BYTES = {"c3": (107 * (33.64e6 + 476.31e6) + 21 * (33.97e6 + 477.69e6)) / 16,
-                     "c3_resident": 8 * (33.64e6 + 476.31e6), "c3_two_pass": 8 * (33.97e6 + 477.69e6),
+NCU_TRAFFIC_BYTES = {"c3": (107 * (33.66e6 + 476.56e6) + 21 * (33.97e6 + 477.98e6)) / 16,
+                     "c3_resident": 8 * (33.66e6 + 476.56e6), "c3_two_pass": 8 * (33.97e6 + 477.98e6),
                      "c4": 4 * (268.45e6 + 98.18e6)}
 
 
