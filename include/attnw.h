@@ -70,6 +70,9 @@ int attnw_fused_f32(const void* Q, const void* K, void* P, int B, int H, int N, 
  *      memory and exchanges local row maxima and sums across CTAs, as the fused kernel of Section VII
  *      does across Tensix cores; serves bfloat16 P and N <= 8192, any other call then returns
  *      ATTNW_ERR_UNSUPPORTED
+ *   3  the same kernel with the exchange the paper leaves as future work (Section IX): the rows are dealt out to
+ *      the CTAs of the cluster, the owner of a row receives its local maxima and sums, reduces them once and
+ *      sends the global values to every CTA (reduce and broadcast) instead of every CTA reducing redundantly
  * Returns ATTNW_ERR_BAD_SHAPE for any other value.
  */
 int attnw_set_fused_variant(int variant);

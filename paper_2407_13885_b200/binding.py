@@ -67,11 +67,12 @@ def version() -> int:
     return int(lib.attnw_version())
 
 
-FUSED_VARIANTS = {"auto": 0, "two_pass": 1, "resident": 2}
+FUSED_VARIANTS = {"auto": 0, "two_pass": 1, "resident": 2, "resident_owner": 3}
 
 
 def set_fused_variant(variant: str | int) -> None:
-    """Selects the kernel behind ``attnw_fused``: "auto" (by shape), "two_pass" or "resident"."""
+    """Selects the kernel behind ``attnw_fused``: "auto" (by shape), "two_pass", "resident" or "resident_owner"
+    (the resident kernel with the reduce-and-broadcast exchange)."""
     code = FUSED_VARIANTS[variant] if isinstance(variant, str) else int(variant)
     _check(lib.attnw_set_fused_variant(code), "attnw_set_fused_variant")
 

@@ -24,7 +24,7 @@ constexpr int kMaxDevices = 64;
 constexpr int kVersion = 100;  // 0.1.0
 
 std::atomic<long long> g_launches{0};
-std::atomic<int> g_fused_variant{0};  // 0 = choose by shape, 1 = two-pass, 2 = SRAM-resident
+std::atomic<int> g_fused_variant{0};  // 0 = choose by shape, 1 = two-pass, 2 = SRAM-resident, 3 = SRAM-resident, owner-reduce exchange
 constexpr double kTwoPassPerSm = 0.9;  // measured: per-SM throughput of the two-pass kernel relative to the resident one
 std::mutex g_mutex;
 
@@ -205,11 +205,11 @@ int launch_fused(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH,
 
 // How many clusters of `cluster_ctas` CTAs of the resident kernel the device can hold at once (cached).
 template <int D, int CMAX>
-int resident_max_clusters_impl(DeviceInfo* dev, int cluster_ctas) {
+int resident_max_clusters_impl(DeviceInfo* dev, int cluster_ctas) {  // (both exchange forms have the same footprint)
     int& cached = dev->resident_clusters[D == 128 ? 1 : 0][cluster_ctas];
     if (cached != 0) return cached;
     using L = ResidentSmem<D, CMAX>;
-    auto kernel = attnw_resident_kernel<D, CMAX>;
+    auto kernel = attnw_resident_kernel<D, CMAX, false>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess ||
         (CMAX > 8 && cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)) {
         (void)cudaGetLastError();
@@ -242,11 +242,11 @@ int resident_max_clusters(DeviceInfo* dev, int cluster_ctas) {
 
 // SRAM-resident single-pass kernel: one cluster of ceil(N / 512) CTAs per 128-row block, persistent over
 // a list of row blocks.  Returns ATTNW_ERR_UNSUPPORTED when the device cannot co-schedule such a cluster.
-template <int D, int CMAX>
+template <int D, int CMAX, bool OWNER>
 int launch_resident_impl(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH, int N, float scale,
                          cudaStream_t stream) {
     using L = ResidentSmem<D, CMAX>;
-    auto kernel = attnw_resident_kernel<D, CMAX>;
+    auto kernel = attnw_resident_kernel<D, CMAX, OWNER>;
     CUtensorMap tm_q, tm_k, tm_p;
     int rc = encode_3d(&tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Q, D, N, BH, 64, kTile);
     if (rc == ATTNW_OK) rc = encode_3d(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, K, D, N, BH, 64, kTile);
@@ -288,9 +288,13 @@ int launch_resident_impl(DeviceInfo* dev, const void* Q, const void* K, void* P,
 
 template <int D>
 int launch_resident(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH, int N, float scale,
-                    cudaStream_t stream) {
-    return (N + kSlab - 1) / kSlab <= 8 ? launch_resident_impl<D, 8>(dev, Q, K, P, BH, N, scale, stream)
-                                        : launch_resident_impl<D, 16>(dev, Q, K, P, BH, N, scale, stream);
+                    cudaStream_t stream, bool owner_reduce = false) {
+    const bool small = (N + kSlab - 1) / kSlab <= 8;
+    if (owner_reduce)
+        return small ? launch_resident_impl<D, 8, true>(dev, Q, K, P, BH, N, scale, stream)
+                     : launch_resident_impl<D, 16, true>(dev, Q, K, P, BH, N, scale, stream);
+    return small ? launch_resident_impl<D, 8, false>(dev, Q, K, P, BH, N, scale, stream)
+                 : launch_resident_impl<D, 16, false>(dev, Q, K, P, BH, N, scale, stream);
 }
 
 template <typename OutT>
@@ -305,7 +309,13 @@ int fused_entry(const void* Q, const void* K, void* P, int B, int H, int N, int 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int variant = g_fused_variant.load(std::memory_order_relaxed);
     const bool resident_fits = sizeof(OutT) == 2 && N <= kResidentMaxN;
-    if (variant == 2 && !resident_fits) return ATTNW_ERR_UNSUPPORTED;
+    if ((variant == 2 || variant == 3) && !resident_fits) return ATTNW_ERR_UNSUPPORTED;
+    if (variant == 3) {
+        if constexpr (sizeof(OutT) == 2)
+            return (d == 64) ? launch_resident<64>(dev, Q, K, P, B * H, N, scale, s, true)
+                             : launch_resident<128>(dev, Q, K, P, B * H, N, scale, s, true);
+        return ATTNW_ERR_UNSUPPORTED;
+    }
     // Choice by shape: the resident kernel whenever it can serve the call.  It spreads one 128-row block over the
     // C SMs of a cluster, so it also fills the device when B*H is small (B*H = 1, N = 4096, d = 128: 25 us
     // against 96 us; B*H = 12, N = 2048, d = 64: 37 against 51 us); between B*H = 8 and 16 at N = 4096 the
@@ -578,7 +588,7 @@ int attnw_query_status(void* stream, unsigned int* device_status) {
 }
 
 int attnw_set_fused_variant(int variant) {
-    if (variant < 0 || variant > 2) return ATTNW_ERR_BAD_SHAPE;
+    if (variant < 0 || variant > 3) return ATTNW_ERR_BAD_SHAPE;
     g_fused_variant.store(variant, std::memory_order_relaxed);
     return ATTNW_OK;
 }

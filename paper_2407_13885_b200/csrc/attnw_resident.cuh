@@ -46,11 +46,13 @@ enum : uint32_t {  // wait sites of this kernel (low byte of the status word)
     kSiteResStageFree = 24,
     kSiteResStageFilled = 25,
     kSiteResStat = 26,
+    kSiteResReduce = 27,
 };
 
 
 constexpr int kKStages = 2;        // key sub-tiles in flight in shared memory
 constexpr int kS1Lag = 1;          // sweep 1 of the next row block trails sweep 2 of the current one by this many slots
+constexpr int kOwnerRedSlots = 144; // owner-reduce exchange: >= C * ceil(128 / C) for every C <= 16
 constexpr int kStoreLag = 3;       // stores allowed to be still reading shared memory when the next one is issued
 constexpr int kStageBoxesMax = 6;  // staged store boxes: three per column half, so that about 100 KB of
                                    // stores can be in flight (the write path needs that much to stay busy)
@@ -82,6 +84,7 @@ struct ResidentBarriers {
     uint64_t s_full[kSlots], slot_free[kSlots];
     uint64_t part_full;
     uint64_t x_full[2];
+    uint64_t red_full[2];  // owner-reduce exchange: the pairs of the rows this CTA owns have arrived
     uint64_t stat_full[4];
     uint64_t out_free[kStageBoxesMax], out_filled[kStageBoxesMax];
     uint32_t tmem_base;
@@ -124,7 +127,11 @@ __device__ __forceinline__ float exp2_chunk_inplace(float (&s)[kChunk], uint64_t
 // Work list: item g = (head g / T, row block g % T); cluster c takes items c, c + G, c + 2G, ...  (neighbouring
 // clusters work on neighbouring row blocks of one head, so its keys stay hot in L2).  Every role of every CTA
 // of the cluster walks the same list.
-template <int D, int CMAX>
+// OWNER = false: every CTA receives every CTA's pairs and reduces them itself (redundantly, as the paper's kernel
+// does).  OWNER = true: the alternative the paper names as future work (Section IX): the rows are dealt out to the
+// CTAs (row i belongs to CTA i mod C); the owner receives the C pairs of its rows, reduces them once and sends
+// (M, 1/L) to every CTA - two hops of latency instead of one, C times fewer messages and reductions.
+template <int D, int CMAX, bool OWNER>
 __global__ void __launch_bounds__(kResidentThreads, 1)
 attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                       const __grid_constant__ CUtensorMap tm_p, int N, int total_items, int cluster_ctas,
@@ -162,6 +169,8 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         ptx::mbar_init(&bars->part_full, kSoftmaxWarps);
         ptx::mbar_init(&bars->x_full[0], 1);
         ptx::mbar_init(&bars->x_full[1], 1);
+        ptx::mbar_init(&bars->red_full[0], 1);
+        ptx::mbar_init(&bars->red_full[1], 1);
         for (int q = 0; q < 4; ++q) ptx::mbar_init(&bars->stat_full[q], 1);
         for (int b = 0; b < kStageBoxes; ++b) {
             ptx::mbar_init(&bars->out_free[b], 1);
@@ -406,13 +415,51 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                     const float2 pc = part[c * kTile + row];
                     lc += pc.y * ptx::ex2_approx(pc.x - mc);
                 }
-                if (warp == 0 && lane == 0)  // arm this CTA's receive barrier for the whole cluster's rows
-                    ptx::mbar_expect_tx(&bars->x_full[par], static_cast<uint32_t>(cluster_ctas * kTile * 8));
-                const uint64_t payload = ptx::pack2(mc, lc);
-                const uint32_t slot_addr = xchg_addr + ((par * CMAX + rank) * kTile + row) * 8u;
-                const uint32_t bar_addr = ptx::smem_u32(&bars->x_full[par]);
-                for (int dst = 0; dst < cluster_ctas; ++dst)
-                    ptx::st_async_b64(ptx::map_to_cta(slot_addr, dst), payload, ptx::map_to_cta(bar_addr, dst));
+                if constexpr (!OWNER) {
+                    if (warp == 0 && lane == 0)  // arm this CTA's receive barrier for the whole cluster's rows
+                        ptx::mbar_expect_tx(&bars->x_full[par], static_cast<uint32_t>(cluster_ctas * kTile * 8));
+                    const uint64_t payload = ptx::pack2(mc, lc);
+                    const uint32_t slot_addr = xchg_addr + ((par * CMAX + rank) * kTile + row) * 8u;
+                    const uint32_t bar_addr = ptx::smem_u32(&bars->x_full[par]);
+                    for (int dst = 0; dst < cluster_ctas; ++dst)
+                        ptx::st_async_b64(ptx::map_to_cta(slot_addr, dst), payload, ptx::map_to_cta(bar_addr, dst));
+                } else {
+                    // exchange area, per parity: red[C senders][rows one CTA can own], then res[128 rows]
+                    const int own_stride = (kTile + cluster_ctas - 1) / cluster_ctas;
+                    const int n_own = (kTile - static_cast<int>(rank) + cluster_ctas - 1) / cluster_ctas;  // rows rank, rank + C, ...
+                    const uint32_t red_addr = xchg_addr + par * (kOwnerRedSlots + kTile) * 8u;
+                    const uint32_t res_addr = red_addr + kOwnerRedSlots * 8u;
+                    if (warp == 0 && lane == 0) {  // arm both receive barriers of this row block
+                        ptx::mbar_expect_tx(&bars->red_full[par], static_cast<uint32_t>(n_own * cluster_ctas * 8));
+                        ptx::mbar_expect_tx(&bars->x_full[par], static_cast<uint32_t>(kTile * 8));
+                    }
+                    {   // hop 1: this row's merged pair goes to the CTA that owns the row
+                        const uint32_t owner = static_cast<uint32_t>(row % cluster_ctas), j = static_cast<uint32_t>(row / cluster_ctas);
+                        ptx::st_async_b64(ptx::map_to_cta(red_addr + (rank * own_stride + j) * 8u, owner), ptx::pack2(mc, lc),
+                                          ptx::map_to_cta(ptx::smem_u32(&bars->red_full[par]), owner));
+                    }
+                    // hop 2: reduce the rows this CTA owns, one thread per (owned row, destination CTA)
+                    ok = __all_sync(0xffffffffu, fused_wait(&bars->red_full[par], (item >> 1) & 1u, abort_flag, kSiteResReduce));
+                    if (!ok) return;
+                    const float2* red = reinterpret_cast<const float2*>(smem + L::kXchgOff) + par * (kOwnerRedSlots + kTile);
+                    const uint32_t res_bar = ptx::smem_u32(&bars->x_full[par]);
+                    for (int idx = row; idx < n_own * cluster_ctas; idx += kTile) {
+                        const int j = idx / cluster_ctas, dst = idx % cluster_ctas;
+                        float2 pc[CMAX];  // all loads at once; entries beyond the cluster repeat its last CTA
+#pragma unroll
+                        for (int c = 0; c < CMAX; ++c) pc[c] = red[((c < cluster_ctas) ? c : cluster_ctas - 1) * own_stride + j];
+                        float m_row = pc[0].x;
+#pragma unroll
+                        for (int c = 1; c < CMAX; ++c) m_row = fmaxf(m_row, pc[c].x);
+                        float l_row = 0.0f;
+#pragma unroll
+                        for (int c = 0; c < CMAX; ++c)
+                            l_row += (c < cluster_ctas) ? pc[c].y * ptx::ex2_approx(pc[c].x - m_row) : 0.0f;
+                        const uint32_t i = static_cast<uint32_t>(j * cluster_ctas) + rank;
+                        ptx::st_async_b64(ptx::map_to_cta(res_addr + i * 8u, dst), ptx::pack2(m_row, 1.0f / l_row),
+                                          ptx::map_to_cta(res_bar, dst));
+                    }
+                }
             }
             if (stamp) ATTNW_STAMP(3, item);
         };
@@ -445,18 +492,24 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                 ok = __all_sync(0xffffffffu, fused_wait(&bars->x_full[par], (item_n >> 1) & 1u, abort_flag, kSiteResExchange));
                 if (!ok) break;
                 if (stamp) ATTNW_STAMP(4, item_n);
-                // all eight exchange slots are read at once (independent loads); slots beyond the cluster are ignored
-                float2 pc[CMAX];
+                if constexpr (!OWNER) {
+                    // all exchange slots are read at once (independent loads); slots beyond the cluster are ignored
+                    float2 pc[CMAX];
 #pragma unroll
-                for (int c = 0; c < CMAX; ++c) pc[c] = xchg[(par * CMAX + c) * kTile + row];
-                m_row = pc[0].x;
+                    for (int c = 0; c < CMAX; ++c) pc[c] = xchg[(par * CMAX + c) * kTile + row];
+                    m_row = pc[0].x;
 #pragma unroll
-                for (int c = 1; c < CMAX; ++c) m_row = (c < cluster_ctas) ? fmaxf(m_row, pc[c].x) : m_row;
-                float l_row = 0.0f;
+                    for (int c = 1; c < CMAX; ++c) m_row = (c < cluster_ctas) ? fmaxf(m_row, pc[c].x) : m_row;
+                    float l_row = 0.0f;
 #pragma unroll
-                for (int c = 0; c < CMAX; ++c)
-                    l_row += (c < cluster_ctas) ? pc[c].y * ptx::ex2_approx(pc[c].x - m_row) : 0.0f;
-                inv_l = 1.0f / l_row;
+                    for (int c = 0; c < CMAX; ++c)
+                        l_row += (c < cluster_ctas) ? pc[c].y * ptx::ex2_approx(pc[c].x - m_row) : 0.0f;
+                    inv_l = 1.0f / l_row;
+                } else {
+                    const float2 ml = xchg[par * (kOwnerRedSlots + kTile) + kOwnerRedSlots + row];  // the owner's (M, 1/L)
+                    m_row = ml.x;
+                    inv_l = ml.y;
+                }
                 stat[row] = make_float2(m_row, inv_l);
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&bars->stat_full[quarter]);

@@ -54,12 +54,13 @@ RESIDENT_SHAPES = [(1, 1, 128, 64), (1, 1, 512, 128), (1, 2, 1024, 128), (1, 3, 
                    (1, 1, 3080, 64), (3, 5, 640, 128), (1, 1, 4608, 64), (1, 1, 5000, 128), (1, 2, 8192, 64)]
 
 
+@pytest.mark.parametrize("variant", ["resident", "resident_owner"])
 @pytest.mark.parametrize("B,H,N,d", RESIDENT_SHAPES)
-def test_resident_variant_matches_oracle(attnw, B, H, N, d):
+def test_resident_variant_matches_oracle(attnw, B, H, N, d, variant):
     q, k = small_fused_inputs(B, H, N, d, stream=N + d + 7)
     scale = float(np.float32(1.0 / math.sqrt(d)))
-    P = run_fused(attnw, q, k, scale, torch.bfloat16, variant="resident")
-    assert_close_to_oracle(P, oracle.attnw(q, k, scale), f"resident B{B} H{H} N{N} d{d}")
+    P = run_fused(attnw, q, k, scale, torch.bfloat16, variant=variant)
+    assert_close_to_oracle(P, oracle.attnw(q, k, scale), f"{variant} B{B} H{H} N{N} d{d}")
 
 
 def test_default_choice_splits_a_call_over_both_kernels(attnw):
