@@ -56,8 +56,11 @@ def _load():
             lib.oracle_attnw_rows.argtypes = [vp, vp, vp, c_long, c_long, c_long, c_long, c_float,
                                               vp, c_long, c_int]
             lib.oracle_scores_rows.argtypes = [vp, vp, vp, c_long, c_long, c_long, c_long, vp, c_long]
+            lib.oracle_attn.argtypes = [vp, vp, vp, vp, c_long, c_long, c_long, c_long, c_float, c_int]
+            lib.oracle_attn_rows.argtypes = [vp, vp, vp, vp, c_long, c_long, c_long, c_long, c_float,
+                                             vp, c_long, c_int]
             for f in (lib.oracle_softmax_rows, lib.oracle_softmax_rows_subset, lib.oracle_attnw,
-                      lib.oracle_attnw_rows, lib.oracle_scores_rows):
+                      lib.oracle_attnw_rows, lib.oracle_scores_rows, lib.oracle_attn, lib.oracle_attn_rows):
                 f.restype = c_int
             lib.paper_cpu_softmax_caching_f32.argtypes = [vp, vp, c_long, c_long]
             lib.paper_cpu_softmax_recomputing_f32.argtypes = [vp, vp, c_long, c_long]
@@ -142,6 +145,27 @@ def attnw_rows(Q, K, scale: float, row_ids, threads: int | None = None) -> np.nd
                                      float(np.float32(scale)), _ptr(ids), ids.size,
                                      threads or host_cores()), "attnw_rows")
     return P
+
+
+def attn(Q, K, V, scale: float, row_ids=None, threads: int | None = None) -> np.ndarray:
+    """``softmax(scale * Q K^T) V`` (Section IV) for bf16 bit patterns ``Q, K, V [B,H,N,d]`` -> float64
+    ``[B,H,N,d]``, or ``[len(row_ids), d]`` for the listed global rows ``(b*H + h)*N + i``."""
+    Q = _as_bf16_bits(Q, "Q")
+    K = _as_bf16_bits(K, "K")
+    V = _as_bf16_bits(V, "V")
+    if Q.shape != K.shape or Q.shape != V.shape or Q.ndim != 4:
+        raise ValueError("Q, K and V must all be [B,H,N,d]")
+    B, H, N, d = Q.shape
+    if row_ids is None:
+        O = np.empty((B, H, N, d), dtype=np.float64)
+        _check(_load().oracle_attn(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), B, H, N, d, float(np.float32(scale)),
+                                   threads or host_cores()), "attn")
+        return O
+    ids = np.ascontiguousarray(row_ids, dtype=np.int64)
+    O = np.empty((ids.size, d), dtype=np.float64)
+    _check(_load().oracle_attn_rows(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), B, H, N, d, float(np.float32(scale)),
+                                    _ptr(ids), ids.size, threads or host_cores()), "attn_rows")
+    return O
 
 
 def scores_rows(Q, K, row_ids) -> np.ndarray:

@@ -28,11 +28,17 @@
  *   - max subtraction is always applied;
  *   - the output is double and is never rounded to a narrower type here.
  *
+ *   attention   O_ic = sum_j P_ij * V_jc                 (Section IV: Attention(Q,K,V) =
+ *                                                         softmax(Q K^T / sqrt(d_k)) V)
+ *
  * Parity pins (tests/test_oracle_pins.py): rows sum to 1 and lie in [0,1];
  * identical keys give exactly 1/N; permuting keys permutes columns; shift
  * invariance (Eq. 1); two-key logistic closed form; geometric-series closed
  * form; one-hot limit; 4x4 brute force of the un-shifted definition in long
- * double; float64 library softmax on the same decoded inputs.
+ * double; float64 library softmax on the same decoded inputs.  For the product
+ * with V: V of ones gives ones; unit-vector columns of V give column sums of P;
+ * identical keys give the mean of V; a single key gives that key's V; linearity
+ * in V; 4x4 brute force in long double; float64 library softmax times V.
  *
  * Rows are independent (Section VI), so threads split rows statically and
  * nothing else is parallelised.
@@ -234,6 +240,71 @@ int oracle_attnw_rows(const uint16_t *Q, const uint16_t *K, double *P, long B, l
             return -3;
     attn_ctx c = {Q, K, P, N, d, (double)scale, row_ids};
     return for_each_row(attn_one, &c, n_ids, N + d, nthreads);
+}
+
+/* ---- attention O = softmax(scale * Q K^T) V (Section IV) ------------------------------
+ * One output row: the row of weights as above, then the weighted sum of the value vectors,
+ * c ascending inside j ascending, all in double. */
+
+typedef struct {
+    attn_ctx a;        /* P is unused here */
+    const uint16_t *V; /* [B*H, N, d] bfloat16 bit patterns */
+    double *O;         /* one row of d doubles per listed row */
+} attnv_ctx;
+
+static void attnv_one(void *vctx, long r, double *scratch)
+{
+    attnv_ctx *c = (attnv_ctx *)vctx;
+    long N = c->a.N, d = c->a.d;
+    long g = c->a.row_ids ? c->a.row_ids[r] : r;
+    long bh = g / N;
+    const uint16_t *q = c->a.Q + (size_t)g * (size_t)d;
+    const uint16_t *Kh = c->a.K + (size_t)bh * (size_t)N * (size_t)d;
+    const uint16_t *Vh = c->V + (size_t)bh * (size_t)N * (size_t)d;
+    double *qd = scratch;         /* d decoded query values */
+    double *z = scratch + d;      /* N scaled scores        */
+    double *p = scratch + d + N;  /* N weights              */
+    double *o = c->O + (size_t)r * (size_t)d;
+    for (long t = 0; t < d; ++t)
+        qd[t] = bf16_to_double(q[t]);
+    for (long j = 0; j < N; ++j) {
+        const uint16_t *k = Kh + (size_t)j * (size_t)d;
+        double s = 0.0;
+        for (long t = 0; t < d; ++t)
+            s += qd[t] * bf16_to_double(k[t]);
+        z[j] = c->a.scale * s;
+    }
+    softmax_row_f64(z, p, N);
+    for (long t = 0; t < d; ++t)
+        o[t] = 0.0;
+    for (long j = 0; j < N; ++j) {
+        const uint16_t *v = Vh + (size_t)j * (size_t)d;
+        for (long t = 0; t < d; ++t)
+            o[t] += p[j] * bf16_to_double(v[t]);
+    }
+}
+
+/* Q, K, V: [B, H, N, d] bfloat16 bits.  O: [B, H, N, d] double. */
+int oracle_attn(const uint16_t *Q, const uint16_t *K, const uint16_t *V, double *O, long B, long H, long N,
+                long d, float scale, int nthreads)
+{
+    if (!Q || !K || !V || !O || B < 1 || H < 1 || N < 1 || d < 1)
+        return -2;
+    attnv_ctx c = {{Q, K, NULL, N, d, (double)scale, NULL}, V, O};
+    return for_each_row(attnv_one, &c, B * H * N, 2 * N + d, nthreads);
+}
+
+/* Only the listed global rows (bh * N + i); O is n_ids x d. */
+int oracle_attn_rows(const uint16_t *Q, const uint16_t *K, const uint16_t *V, double *O, long B, long H,
+                     long N, long d, float scale, const long *row_ids, long n_ids, int nthreads)
+{
+    if (!Q || !K || !V || !O || !row_ids || B < 1 || H < 1 || N < 1 || d < 1 || n_ids < 1)
+        return -2;
+    for (long r = 0; r < n_ids; ++r)
+        if (row_ids[r] < 0 || row_ids[r] >= B * H * N)
+            return -3;
+    attnv_ctx c = {{Q, K, NULL, N, d, (double)scale, row_ids}, V, O};
+    return for_each_row(attnv_one, &c, n_ids, 2 * N + d, nthreads);
 }
 
 /* Raw (unscaled) scores of the listed rows, for tests that look at one step alone. */

@@ -283,3 +283,82 @@ def test_row_partition_golden():
         assert inputs.shard_range(units, 0, workers)[0] == 0
         for r in range(workers - 1):
             assert inputs.shard_range(units, r, workers)[1] == inputs.shard_range(units, r + 1, workers)[0]
+
+
+# ---- the product with V: Attention(Q, K, V) of Section IV --------------------------------
+
+def rand_v(B, H, N, d, sigma=1.0, stream=500):
+    return inputs.normal_bf16_bits(7, stream, B * H * N * d, sigma).reshape(B, H, N, d)
+
+
+def test_attention_of_constant_values_is_that_constant():
+    q, k = rand_qk(1, 2, 50, 64, stream=510)
+    v = bits(np.full((1, 2, 50, 64), 1.5, dtype=np.float32))
+    O = oracle.attn(q, k, v, 0.125)
+    assert np.max(np.abs(O - 1.5)) <= 1e-14          # rows of P sum to one
+
+
+def test_attention_with_unit_vector_values_gives_column_sums_of_the_weights():
+    N, d = 40, 8
+    q, k = rand_qk(1, 1, N, d, stream=520)
+    vv = np.zeros((1, 1, N, d), dtype=np.float32)
+    for j in range(N):
+        vv[0, 0, j, j % d] = 1.0
+    O = oracle.attn(q, k, bits(vv), 0.3)[0, 0]
+    P = oracle.attnw(q, k, 0.3)[0, 0]
+    for c in range(d):
+        assert np.max(np.abs(O[:, c] - P[:, c::d].sum(axis=1))) <= 1e-14
+
+
+def test_attention_with_identical_keys_is_the_mean_value_and_single_key_is_its_value():
+    N, d = 64, 16
+    q, _ = rand_qk(1, 1, N, d, stream=530)
+    key = inputs.normal_bf16_bits(5, 5, d, 1.0)
+    kk = np.broadcast_to(key, (1, 1, N, d)).copy()
+    vals = (np.arange(N * d).reshape(1, 1, N, d) % 17 - 8).astype(np.float32) / 4.0   # exact in bf16
+    O = oracle.attn(q, kk, bits(vals), 0.7)[0, 0]
+    assert np.max(np.abs(O - vals[0, 0].astype(np.float64).mean(axis=0))) <= 1e-13
+    q1, k1 = rand_qk(1, 1, 1, d, stream=531)
+    v1 = rand_v(1, 1, 1, d, stream=532)
+    assert np.array_equal(oracle.attn(q1, k1, v1, 0.25)[0, 0, 0], dec(v1)[0, 0, 0])
+
+
+def test_attention_is_linear_in_the_values():
+    q, k = rand_qk(1, 1, 30, 32, stream=540)
+    a = (np.random.default_rng(1).integers(-16, 17, size=(1, 1, 30, 32)) / 8.0).astype(np.float32)
+    b = (np.random.default_rng(2).integers(-16, 17, size=(1, 1, 30, 32)) / 8.0).astype(np.float32)
+    Oa, Ob = oracle.attn(q, k, bits(a), 0.2), oracle.attn(q, k, bits(b), 0.2)
+    Oab = oracle.attn(q, k, bits(a + 2 * b), 0.2)     # a + 2b stays exact in bf16 (multiples of 1/8 below 8)
+    assert np.max(np.abs(Oab - (Oa + 2 * Ob))) <= 1e-13
+
+
+def test_attention_brute_force_4x4_long_double():
+    rng = np.random.default_rng(77)
+    ld = np.longdouble
+    for trial in range(20):
+        N, d = 4, 4
+        qv = (rng.integers(-8, 9, size=(N, d)) / 4.0).astype(np.float32)
+        kv = (rng.integers(-8, 9, size=(N, d)) / 4.0).astype(np.float32)
+        vv = (rng.integers(-8, 9, size=(N, d)) / 4.0).astype(np.float32)
+        scale = np.float32(0.5)
+        O = oracle.attn(bits(qv.reshape(1, 1, N, d)), bits(kv.reshape(1, 1, N, d)), bits(vv.reshape(1, 1, N, d)),
+                        float(scale))[0, 0]
+        for i in range(N):
+            e = [np.exp(ld(scale) * sum(ld(qv[i, c]) * ld(kv[j, c]) for c in range(d))) for j in range(N)]
+            tot = sum(e)
+            for c in range(d):
+                want = sum(e[j] / tot * ld(vv[j, c]) for j in range(N))
+                assert abs(float(want) - O[i, c]) <= 1e-13
+
+
+@pytest.mark.parametrize("shape,sigma", [((1, 2, 100, 64), 1.0), ((2, 1, 77, 128), 4.0)])
+def test_attention_against_float64_library(shape, sigma):
+    q, k = rand_qk(*shape, sigma=sigma, stream=550)
+    v = rand_v(*shape, stream=552)
+    scale = float(np.float32(1.0 / math.sqrt(shape[3])))
+    O = oracle.attn(q, k, v, scale)
+    Z = scale * np.einsum("bhic,bhjc->bhij", dec(q), dec(k))
+    ref = np.einsum("bhij,bhjc->bhic", scipy.special.softmax(Z, axis=-1), dec(v))
+    assert np.max(np.abs(O - ref)) <= 1e-12
+    ids = [0, 5, shape[0] * shape[1] * shape[2] - 1]
+    assert np.array_equal(oracle.attn(q, k, v, scale, row_ids=ids), O.reshape(-1, shape[3])[ids])
