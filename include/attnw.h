@@ -1,8 +1,9 @@
 /*
  * attnw - attention weights P = Softmax(scale * Q K^T) on NVIDIA B200 (sm_100a).
  *
- * C ABI of libattnw.so.  Two operations, each a hand-written CUDA kernel:
+ * C ABI of libattnw.so.  The operations, each a hand-written CUDA kernel:
  *
+ *   attn_fused     the whole of Attention(Q, K, V) = softmax(Q K^T / sqrt(d_k)) V of Section IV in one kernel
  *   attnw_fused*   matmul + scaling + Softmax in one kernel; scores never reach HBM
  *                  (the fused kernel of Section VII of "Attention in SRAM on Tenstorrent
  *                  Grayskull"; the product is Attention's softmax(QK^T/sqrt(d_k)) of Section IV).
@@ -56,6 +57,20 @@ typedef enum attnw_status {
  */
 int attnw_fused(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream);
 int attnw_fused_f32(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream);
+
+/*
+ * attn_fused: O[b,h,i,c] = sum_j P[b,h,i,j] * V[b,h,j,c] with P as defined for attnw_fused - Attention(Q, K, V) of
+ * Section IV, the product with V that Section IX leaves as future work - in one kernel; neither the scores nor the
+ * weights reach HBM.
+ *
+ *   Q, K, V  device, bfloat16, [B, H, N, d]                    (read only)
+ *   O        device, bfloat16, [B, H, N, d]; every element is written exactly once; must not overlap Q, K or V
+ *   B,H,N    >= 1 (no divisibility condition on N);  d in {64, 128};  scale finite, >= 0
+ * Scores and the products with V are accumulated in float32 on the tensor cores; max, exponentials and sums are
+ * float32; the weights enter the second product rounded to bfloat16 (nearest even), O is rounded to bfloat16.
+ */
+int attn_fused(const void* Q, const void* K, const void* V, void* O, int B, int H, int N, int d, float scale,
+               void* stream);
 
 /*
  * Which kernel attnw_fused uses (process-wide; the results are the same within the stated tolerances):

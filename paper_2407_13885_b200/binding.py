@@ -17,6 +17,7 @@ _vp, _int, _ll, _float = ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong, ctype
 
 # name -> (restype, argtypes); mirrors include/attnw.h one to one
 SIGNATURES = {
+    "attn_fused": (_int, [_vp, _vp, _vp, _vp, _int, _int, _int, _int, _float, _vp]),
     "attnw_fused": (_int, [_vp, _vp, _vp, _int, _int, _int, _int, _float, _vp]),
     "attnw_fused_f32": (_int, [_vp, _vp, _vp, _int, _int, _int, _int, _float, _vp]),
     "softmax_rows": (_int, [_vp, _vp, _ll, _ll, _vp]),
@@ -123,6 +124,27 @@ def attnw_fused(Q: torch.Tensor, K: torch.Tensor, scale: float, P: torch.Tensor 
         _check(fn(Q.data_ptr(), K.data_ptr(), P.data_ptr(), B, H, N, d, float(scale), _stream_ptr(stream)),
                "attnw_fused")
     return P
+
+
+def attn_fused(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, scale: float, O: torch.Tensor | None = None,
+               stream=None) -> torch.Tensor:
+    """``O = Softmax(scale * Q K^T) V`` in one fused kernel; ``Q, K, V, O``: CUDA bfloat16 ``[B, H, N, d]``.
+    Asynchronous on ``stream`` (default: torch's current stream)."""
+    for t, name in ((Q, "Q"), (K, "K"), (V, "V")):
+        _require_cuda(t, name, torch.bfloat16)
+    if Q.dim() != 4 or Q.shape != K.shape or Q.shape != V.shape:
+        raise ValueError("Q, K and V must all be [B, H, N, d]")
+    B, H, N, d = Q.shape
+    if O is None:
+        O = torch.empty((B, H, N, d), dtype=torch.bfloat16, device=Q.device)
+    else:
+        _require_cuda(O, "O", torch.bfloat16)
+        if tuple(O.shape) != (B, H, N, d):
+            raise ValueError("O must be [B, H, N, d]")
+    with torch.cuda.device(Q.device):
+        _check(lib.attn_fused(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), B, H, N, d, float(scale),
+                              _stream_ptr(stream)), "attn_fused")
+    return O
 
 
 def softmax_rows(S: torch.Tensor, P: torch.Tensor | None = None, out_dtype: torch.dtype = torch.bfloat16,

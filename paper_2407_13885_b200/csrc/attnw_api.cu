@@ -13,6 +13,7 @@
 
 #include "../../include/attnw.h"
 #include "attnw_fused.cuh"
+#include "attn_fused.cuh"
 #include "attnw_resident.cuh"
 #include "softmax_rows.cuh"
 
@@ -297,6 +298,45 @@ int launch_resident(DeviceInfo* dev, const void* Q, const void* K, void* P, int 
                  : launch_resident_impl<D, 16, false>(dev, Q, K, P, BH, N, scale, stream);
 }
 
+template <int D>
+int launch_attn(const void* Q, const void* K, const void* V, void* O, int BH, int N, float scale, cudaStream_t stream) {
+    using L = FusedSmem<D>;
+    auto kernel = av::attn_fused_kernel<D>;
+    CUtensorMap tm_q, tm_k, tm_v, tm_o;
+    int rc = encode_3d(&tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Q, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, K, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, V, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_o, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, O, D, N, BH, 64, kTile);
+    if (rc != ATTNW_OK) return rc;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    const int row_blocks = (N + kRowsPerCta - 1) / kRowsPerCta;
+    const float scale_log2e = static_cast<float>(static_cast<double>(scale) * 1.4426950408889634074);
+    kernel<<<static_cast<unsigned>(BH * row_blocks), kFusedThreads, L::kDynamicBytes, stream>>>(tm_q, tm_k, tm_v, tm_o, N,
+                                                                                                 row_blocks, scale_log2e);
+    if (cudaGetLastError() != cudaSuccess) return ATTNW_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTNW_OK;
+}
+
+// Host-only checks of the attention call; no CUDA call is made here.
+int validate_attn(const void* Q, const void* K, const void* V, const void* O, int B, int H, int N, int d, float scale) {
+    if (!Q || !K || !V || !O) return ATTNW_ERR_NULL_POINTER;
+    if (B < 1 || H < 1 || N < 1 || d < 1) return ATTNW_ERR_BAD_SHAPE;
+    if (!(scale >= 0.0f) || !std::isfinite(scale)) return ATTNW_ERR_BAD_SHAPE;
+    const long long bh = static_cast<long long>(B) * H;
+    if (bh > INT_MAX) return ATTNW_ERR_BAD_SHAPE;
+    if (bh * ((static_cast<long long>(N) + kRowsPerCta - 1) / kRowsPerCta) > INT_MAX) return ATTNW_ERR_BAD_SHAPE;
+    if (N > (1 << 24)) return ATTNW_ERR_BAD_SHAPE;
+    if (d != 64 && d != 128) return ATTNW_ERR_UNSUPPORTED;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return ATTNW_ERR_MISALIGNED;
+    const unsigned long long bytes = static_cast<unsigned long long>(bh) * N * d * 2ull;
+    if (overlaps(O, bytes, Q, bytes) || overlaps(O, bytes, K, bytes) || overlaps(O, bytes, V, bytes)) return ATTNW_ERR_ALIASING;
+    return ATTNW_OK;
+}
+
 template <typename OutT>
 int fused_entry(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream) {
     int rc = validate_fused(Q, K, P, B, H, N, d, scale, sizeof(OutT));
@@ -459,6 +499,19 @@ constexpr unsigned long long kHostChunkBytes = 256ull << 20;  // target size of 
 }  // namespace
 
 extern "C" {
+
+int attn_fused(const void* Q, const void* K, const void* V, void* O, int B, int H, int N, int d, float scale,
+               void* stream) {
+    int rc = validate_attn(Q, K, V, O, B, H, N, d, scale);
+    if (rc != ATTNW_OK) return rc;
+    DeviceInfo* dev = nullptr;
+    rc = current_device(&dev);
+    if (rc != ATTNW_OK) return rc;
+    rc = load_encoder();
+    if (rc != ATTNW_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    return d == 64 ? launch_attn<64>(Q, K, V, O, B * H, N, scale, s) : launch_attn<128>(Q, K, V, O, B * H, N, scale, s);
+}
 
 int attnw_fused(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream) {
     return fused_entry<__nv_bfloat16>(Q, K, P, B, H, N, d, scale, stream);

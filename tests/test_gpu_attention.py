@@ -1,0 +1,104 @@
+"""attn_fused (Attention(Q, K, V) of Section IV in one kernel) on the GPU against the fp64 oracle, through the C ABI."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import bits_to_cuda_bf16, small_fused_inputs
+from paper_2407_13885_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def attnw():
+    from paper_2407_13885_b200 import binding
+    return binding
+
+
+def rand_v(B, H, N, d, sigma=1.0, stream=900):
+    return inputs.normal_bf16_bits(11, stream, B * H * N * d, sigma).reshape(B, H, N, d)
+
+
+def run_attn(attnw, q, k, v, scale):
+    B, H, N, d = q.shape
+    # guard rows before and after O: the kernel must write O and nothing else
+    raw = torch.full((B * H * N * d + 2 * 4096,), float("nan"), dtype=torch.bfloat16, device="cuda")
+    O = raw[4096:4096 + B * H * N * d].view(B, H, N, d)
+    attnw.attn_fused(bits_to_cuda_bf16(q), bits_to_cuda_bf16(k), bits_to_cuda_bf16(v), scale, O=O)
+    torch.cuda.synchronize()
+    assert attnw.query_status() == 0
+    assert bool(torch.isnan(raw[:4096]).all()) and bool(torch.isnan(raw[-4096:]).all())
+    return O
+
+
+def tolerance(v_bits):
+    # The weights enter the second product rounded to bf16 (relative 2^-9 each, and they sum to one), O is rounded
+    # to bf16 (relative 2^-9, |O| <= max|V|): |O_gpu - O| <= 2^-9 max|V| + 2^-9 max|V|, plus float32 dust.
+    return 2.0 ** -8 * float(np.abs(inputs.bf16_bits_to_f32(v_bits)).max()) + 1e-5
+
+
+SHAPES = [(1, 1, 128, 64), (1, 1, 128, 128), (1, 2, 256, 64), (2, 1, 384, 128), (1, 3, 512, 64), (1, 1, 8, 64),
+          (1, 2, 72, 128), (1, 1, 136, 64), (2, 2, 200, 128), (1, 1, 264, 64), (1, 1, 1000, 128), (1, 1, 1160, 64),
+          (1, 1, 1, 64), (1, 1, 77, 128)]
+
+
+@pytest.mark.parametrize("B,H,N,d", SHAPES)
+def test_attention_matches_oracle(attnw, B, H, N, d):
+    q, k = small_fused_inputs(B, H, N, d, stream=N + d + 3)
+    v = rand_v(B, H, N, d, stream=N + d + 5)
+    scale = float(np.float32(1.0 / math.sqrt(d)))
+    O = run_attn(attnw, q, k, v, scale)
+    ref = oracle.attn(q, k, v, scale)
+    got = O.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all()
+    assert np.max(np.abs(got - ref)) <= tolerance(v), (np.max(np.abs(got - ref)), tolerance(v))
+
+
+def test_attention_large_logits(attnw):
+    q, k = small_fused_inputs(1, 2, 1024, 128, sigma=4.0, stream=61)
+    v = rand_v(1, 2, 1024, 128, stream=62)
+    scale = float(np.float32(1.0 / math.sqrt(128.0)))
+    O = run_attn(attnw, q, k, v, scale)
+    ref = oracle.attn(q, k, v, scale)
+    got = O.float().cpu().numpy().astype(np.float64)
+    # At sigma = 4 the raw scores reach ~1e3 and the tensor cores' float32 accumulation error of a score,
+    # (d/16) * 17 * 2^-24 * max|s|, is no longer dust: dp <= p * scale * ds for every weight of a row, and a
+    # perturbed row moves that much weight from some keys to others, so dO <= 2 * scale * ds * max|V| on top.
+    s_abs = float(np.max(np.abs(oracle.scores_rows(q, k, np.arange(2 * 1024)))))
+    v_abs = float(np.abs(inputs.bf16_bits_to_f32(v)).max())
+    tol = tolerance(v) + 2.0 * scale * s_abs * (128 / 16) * 17 * 2.0 ** -24 * v_abs
+    err = float(np.max(np.abs(got - ref)))
+    assert err <= tol, f"{err:.3e} > {tol:.3e}"
+
+
+def test_attention_of_constant_and_unit_vector_values(attnw):
+    # constant V: O is that constant (rows of the weights sum to one)
+    q, k = small_fused_inputs(1, 2, 520, 128, stream=71)
+    ones = inputs.f32_to_bf16_bits(np.full((1, 2, 520, 128), 1.5, dtype=np.float32))
+    O = run_attn(attnw, q, k, ones, 0.09)
+    assert float((O.float() - 1.5).abs().max()) <= 1.5 * 2.0 ** -7
+    # V[j, c] = 1 where c == j mod d: column c of O is the sum of the weights of keys j = c (mod d) - catches any
+    # mix-up of the key and feature axes of V
+    N, d = 300, 64
+    q, k = small_fused_inputs(1, 1, N, d, stream=72)
+    vv = np.zeros((1, 1, N, d), dtype=np.float32)
+    for j in range(N):
+        vv[0, 0, j, j % d] = 1.0
+    O = run_attn(attnw, q, k, inputs.f32_to_bf16_bits(vv), 0.125)[0, 0].float().cpu().numpy().astype(np.float64)
+    P = oracle.attnw(q, k, 0.125)[0, 0]
+    want = np.stack([P[:, c::d].sum(axis=1) for c in range(d)], axis=1)
+    assert np.max(np.abs(O - want)) <= 2.0 ** -8
+
+
+def test_attention_argument_errors(attnw):
+    x = torch.zeros((1, 1, 128, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(attnw.AttnwError) as e:
+        attnw.attn_fused(x, x, x, 0.1, O=x)
+    assert e.value.code == 7
+    y = torch.zeros((1, 1, 128, 96), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(attnw.AttnwError) as e:
+        attnw.attn_fused(y, y, y, 0.1)
+    assert e.value.code == 4
