@@ -245,6 +245,26 @@ def secondary_config(binding, inputs, name, peaks, steps=20, warmup=3):
             "steps": steps}
 
 
+def attention_config(binding, inputs, name, peaks, steps=20, warmup=3):
+    """Short kernel-only measurement of attn_fused (the product with V, Section IV) on the shape of one of the
+    configurations, with V drawn like K on its own stream (reported beside the headline, not part of it)."""
+    import torch
+    w = inputs.WORKLOADS[name]
+    q, k = inputs.make_qk(w)
+    v = inputs.normal_bf16_bits(inputs.SEED, 2 * w.cfg_id + 100, w.B * w.H * w.N * w.d, 1.0)
+    as_t = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).reshape(w.B, w.H, w.N, w.d).cuda()  # noqa: E731
+    Q, K, V = as_t(q), as_t(k), as_t(v)
+    O = torch.empty_like(Q)
+    ms = time_launches(lambda: binding.attn_fused(Q, K, V, w.scale, O=O), steps, warmup, torch.cuda.synchronize) / steps
+    flops = 2.0 * w.flops                       # Q K^T and P V, 2 N^2 d multiply-adds each per head
+    bytes_alg = 4 * w.B * w.H * w.N * w.d * 2   # Q, K, V read once, O written once
+    t_flop = flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = bytes_alg / (peaks["hbm_gbs"] * 1e9)
+    return {"op": "attn_fused: O = Softmax(scale Q K^T) V, bf16", "ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+            "roofline_frac": max(t_hbm, t_flop) / (ms * 1e-3), "bound": "tensor" if t_flop >= t_hbm else "hbm",
+            "peak_tflops": peaks["bf16_tflops"], "algorithmic_flops": flops, "steps": steps}
+
+
 def run_profile_case(args):
     """A reduced case of one kernel for profiler captures (`--profile fused|rows`): the same kernel and
     tile configuration as the headline launch on inputs that still exceed the L2 but hold well under a
@@ -264,6 +284,18 @@ def run_profile_case(args):
         P = torch.empty((1, heads, w.N, w.N), dtype=torch.bfloat16, device="cuda")
         fn = lambda: binding.attnw_fused(Q, K, w.scale, P=P)  # noqa: E731
         desc = f"fused B=1 H={heads} N={w.N} d={w.d} (P {w.p_bytes >> 20} MiB)"
+    elif args.profile == "attention":
+        base = inputs.WORKLOADS[args.workload]
+        heads = 16
+        w = inputs.Workload(base.name + "-attention-reduced", "fused", B=1, H=heads, N=base.N, d=base.d, sigma=base.sigma,
+                            scale=base.scale, p_dtype=base.p_dtype, cfg_id=base.cfg_id)
+        q, k = inputs.make_qk(w)
+        v = inputs.normal_bf16_bits(inputs.SEED, 2 * w.cfg_id + 100, heads * w.N * w.d, 1.0)
+        as_t = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).reshape(1, heads, w.N, w.d).cuda()  # noqa: E731
+        Q, K, V = as_t(q), as_t(k), as_t(v)
+        O = torch.empty_like(Q)
+        fn = lambda: binding.attn_fused(Q, K, V, w.scale, O=O)  # noqa: E731
+        desc = f"attn_fused B=1 H={heads} N={w.N} d={w.d}"
     else:
         base = inputs.WORKLOADS["c4"]
         rows = 8192
@@ -427,6 +459,8 @@ def run_ours(args):
         for name in ("c4", "c5", "c2"):
             other[name] = secondary_config(binding, inputs, name, peaks)
             torch.cuda.empty_cache()
+        other["attention_c3"] = attention_config(binding, inputs, "c3", peaks)
+        torch.cuda.empty_cache()
         line["other_configs"] = other
     print(json.dumps(line))
     return 0
@@ -448,7 +482,7 @@ def main():
     ap.add_argument("--sustained-seconds", type=float, default=2.0)
     ap.add_argument("--variant", choices=["auto", "two_pass", "resident"], default="auto",
                     help="kernel behind attnw_fused (see attnw_set_fused_variant)")
-    ap.add_argument("--profile", choices=["fused", "rows"], default=None,
+    ap.add_argument("--profile", choices=["fused", "rows", "attention"], default=None,
                     help="run a reduced case of one kernel for an ncu capture instead of the benchmark")
     args = ap.parse_args()
     if args.impl == "reference":
