@@ -73,6 +73,17 @@ int attn_fused(const void* Q, const void* K, const void* V, void* O, int B, int 
                void* stream);
 
 /*
+ * Which kernel attn_fused uses (process-wide; the results agree within the stated tolerance):
+ *   0  default: the one-pass kernel
+ *   1  two-pass kernel: row maxima and sums in a first pass over the keys, normalised weights times V in a second
+ *      pass that recomputes the score tiles (two exponentials and three MMA passes per element)
+ *   2  one-pass kernel: the online form of Eq. 1 - running row maximum and sum, O rescaled when the maximum has
+ *      grown (one exponential and two MMA passes per element), division by the row sum at the end
+ * Returns ATTNW_ERR_BAD_SHAPE for any other value.
+ */
+int attnw_set_attn_variant(int variant);
+
+/*
  * Which kernel attnw_fused uses (process-wide; the results are the same within the stated tolerances):
  *   0  choose by shape (default): the SRAM-resident kernel when P is bfloat16 and N <= 4096; the
  *      two-pass kernel otherwise (and always for attnw_fused_f32).  Clusters cannot occupy every SM

@@ -27,6 +27,7 @@ SIGNATURES = {
     "attnw_host_release": (_int, []),
     "attnw_query_status": (_int, [_vp, ctypes.POINTER(ctypes.c_uint)]),
     "attnw_set_fused_variant": (_int, [_int]),
+    "attnw_set_attn_variant": (_int, [_int]),
     "attnw_launch_count": (_ll, [_int]),
     "attnw_strerror": (ctypes.c_char_p, [_int]),
     "attnw_version": (_int, []),
@@ -76,6 +77,15 @@ def set_fused_variant(variant: str | int) -> None:
     (the resident kernel with the reduce-and-broadcast exchange)."""
     code = FUSED_VARIANTS[variant] if isinstance(variant, str) else int(variant)
     _check(lib.attnw_set_fused_variant(code), "attnw_set_fused_variant")
+
+
+ATTN_VARIANTS = {"auto": 0, "two_pass": 1, "one_pass": 2}
+
+
+def set_attn_variant(variant: str | int) -> None:
+    """Selects the kernel behind ``attn_fused``: "auto" (the one-pass kernel), "two_pass" or "one_pass"."""
+    code = ATTN_VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    _check(lib.attnw_set_attn_variant(code), "attnw_set_attn_variant")
 
 
 def launch_count(reset: bool = False) -> int:

@@ -14,6 +14,7 @@
 #include "../../include/attnw.h"
 #include "attnw_fused.cuh"
 #include "attn_fused.cuh"
+#include "attn_onepass.cuh"
 #include "attnw_resident.cuh"
 #include "softmax_rows.cuh"
 
@@ -25,6 +26,7 @@ constexpr int kMaxDevices = 64;
 constexpr int kVersion = 100;  // 0.1.0
 
 std::atomic<long long> g_launches{0};
+std::atomic<int> g_attn_variant{0};   // 0 = default (one pass), 1 = two-pass, 2 = one pass
 std::atomic<int> g_fused_variant{0};  // 0 = choose by shape, 1 = two-pass, 2 = SRAM-resident, 3 = SRAM-resident, owner-reduce exchange
 constexpr double kTwoPassPerSm = 0.9;  // measured: per-SM throughput of the two-pass kernel relative to the resident one
 std::mutex g_mutex;
@@ -321,6 +323,29 @@ int launch_attn(const void* Q, const void* K, const void* V, void* O, int BH, in
     return ATTNW_OK;
 }
 
+template <int D>
+int launch_attn_onepass(const void* Q, const void* K, const void* V, void* O, int BH, int N, float scale, cudaStream_t stream) {
+    using L = av1::Smem<D>;
+    auto kernel = av1::attn_onepass_kernel<D>;
+    CUtensorMap tm_q, tm_k, tm_v, tm_o;
+    int rc = encode_3d(&tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Q, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, K, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_v, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, V, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_o, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, O, D, N, BH, 64, kTile);
+    if (rc != ATTNW_OK) return rc;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    const int row_blocks = (N + kRowsPerCta - 1) / kRowsPerCta;
+    const float scale_log2e = static_cast<float>(static_cast<double>(scale) * 1.4426950408889634074);
+    kernel<<<static_cast<unsigned>(BH * row_blocks), av1::kThreads, L::kDynamicBytes, stream>>>(tm_q, tm_k, tm_v, tm_o, N,
+                                                                                                 row_blocks, scale_log2e);
+    if (cudaGetLastError() != cudaSuccess) return ATTNW_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTNW_OK;
+}
+
 // Host-only checks of the attention call; no CUDA call is made here.
 int validate_attn(const void* Q, const void* K, const void* V, const void* O, int B, int H, int N, int d, float scale) {
     if (!Q || !K || !V || !O) return ATTNW_ERR_NULL_POINTER;
@@ -510,7 +535,16 @@ int attn_fused(const void* Q, const void* K, const void* V, void* O, int B, int 
     rc = load_encoder();
     if (rc != ATTNW_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    return d == 64 ? launch_attn<64>(Q, K, V, O, B * H, N, scale, s) : launch_attn<128>(Q, K, V, O, B * H, N, scale, s);
+    if (g_attn_variant.load(std::memory_order_relaxed) == 1)
+        return d == 64 ? launch_attn<64>(Q, K, V, O, B * H, N, scale, s) : launch_attn<128>(Q, K, V, O, B * H, N, scale, s);
+    return d == 64 ? launch_attn_onepass<64>(Q, K, V, O, B * H, N, scale, s)
+                   : launch_attn_onepass<128>(Q, K, V, O, B * H, N, scale, s);
+}
+
+int attnw_set_attn_variant(int variant) {
+    if (variant < 0 || variant > 2) return ATTNW_ERR_BAD_SHAPE;
+    g_attn_variant.store(variant, std::memory_order_relaxed);
+    return ATTNW_OK;
 }
 
 int attnw_fused(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream) {

@@ -97,5 +97,12 @@ def test_fused_variant_knob(lib):
         assert lib.attnw_set_fused_variant(v) == 0
 
 
+def test_attention_variant_knob(lib):
+    assert lib.attnw_set_attn_variant(3) == 2
+    assert lib.attnw_set_attn_variant(-1) == 2
+    for v in (1, 2, 0):
+        assert lib.attnw_set_attn_variant(v) == 0
+
+
 def test_query_status_rejects_null(lib):
     assert lib.attnw_query_status(None, None) == 1
