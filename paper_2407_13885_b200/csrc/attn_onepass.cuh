@@ -3,9 +3,10 @@
 //
 // A CTA owns 256 query rows (two tiles).  Per key tile j and query tile q:
 //   MMA 1     S = Q_q K_j^T                       128 x 128 fp32 in tensor memory (one buffer per query tile)
-//   Softmax   one THREAD per row: all 128 scores of the row go to registers (the buffer is handed back at once, so
-//             the next tile's MMA 1 runs meanwhile); row maximum; p = 2^(c s - mb) with the row's offset mb;
-//             l += sum p; P (bf16) is written to shared memory as a K-major MMA operand
+//   Softmax   two threads per row, 64 columns each: a thread takes its scores to registers (the buffer is handed back
+//             at once, so the next tile's MMA 1 runs meanwhile) and also reads the other thread's 64 columns for
+//             their maximum, so both know the row maximum without an exchange; p = 2^(c s - mb) with the row's
+//             offset mb; l += sum p; P (bf16) is written to shared memory as a K-major MMA operand
 //   MMA 2     O_q += P V_j                        128 x d fp32 in tensor memory; V_j as TMA delivers it
 //             ([128 keys x d], an MN-major B operand)
 // The offset mb of a row follows its running maximum lazily: it moves only when the maximum has grown by more than 8
@@ -19,10 +20,10 @@
 namespace attnw {
 namespace av1 {
 
-constexpr int kSmWarps = 8;       // Softmax warps: query tile (2) x TMEM lane quarter (4); one thread per row
-constexpr int kProducer = 8;
-constexpr int kMma = 9;
-constexpr int kThreads = 320;
+constexpr int kSmWarps = 16;      // Softmax warps: query tile (2) x column half (2) x TMEM lane quarter (4)
+constexpr int kProducer = 16;
+constexpr int kMma = 17;
+constexpr int kThreads = 576;
 constexpr int kStages = 3;        // ring of K / V tiles (128 keys x d)
 constexpr float kLazy = 8.0f;     // the offset follows the maximum only when it has grown by more than this
 
@@ -36,6 +37,7 @@ enum : uint32_t {  // wait sites of this kernel (low byte of the status word)
     kSitePFree = 102,
     kSiteOFull = 103,
     kSiteOutFilled = 104,
+    kSiteLFull = 105,
 };
 
 template <int D>
@@ -56,15 +58,34 @@ static_assert(Smem<128>::kDynamicBytes <= 227 * 1024, "shared memory budget");
 struct Barriers {
     uint64_t q_full;
     uint64_t k_full[kStages], k_empty[kStages];
-    uint64_t s_full[2], s_free[2];  // per query tile: scores written / read into registers (4 warps)
-    uint64_t p_full[2], p_free[2];  // per query tile: P tile written (4 warps) / read by its MMAs
+    uint64_t s_full[2], s_free[2];  // per query tile: scores written / read into registers (8 warps)
+    uint64_t p_full[2], p_free[2];  // per query tile: P tile written (8 warps) / read by its MMAs
     uint64_t o_full;
+    uint64_t l_full[2];      // per query tile: the partial row sums of the 8 warps are in shared memory
     uint64_t out_filled[2];
     uint32_t tmem_base;
     uint32_t abort_flag;
     uint32_t prior_failure;
 };
 static_assert(sizeof(Barriers) <= 256, "barrier block must fit its slot");
+
+// The bounded wait of the other kernels, but expanded in place: where a thread holds a row of scores in registers,
+// a call would spill them around it.
+__device__ __forceinline__ bool wait_in_place(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t site) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t spin = 1;; ++spin) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if ((spin & 63u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitLimitCycles) {
+                *abort_flag = 1;
+                atomicCAS(&g_attnw_status, 0u, 0x80000000u | site);
+                return false;
+            }
+        }
+    }
+}
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -97,10 +118,11 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         for (int q = 0; q < 2; ++q) {
             ptx::mbar_init(&bars->s_full[q], 1);
-            ptx::mbar_init(&bars->s_free[q], 4);
-            ptx::mbar_init(&bars->p_full[q], 4);
+            ptx::mbar_init(&bars->s_free[q], 8);
+            ptx::mbar_init(&bars->p_full[q], 8);
             ptx::mbar_init(&bars->p_free[q], 1);
-            ptx::mbar_init(&bars->out_filled[q], 3);
+            ptx::mbar_init(&bars->l_full[q], 8);
+            ptx::mbar_init(&bars->out_filled[q], 7);
         }
         ptx::mbar_init(&bars->o_full, 1);
         bars->abort_flag = 0;
@@ -189,6 +211,7 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(q * 2 * kTile);
                 const uint32_t a_addr = q_addr + static_cast<uint32_t>(q * L::kTileBytes);
                 if (ptx::elect_one()) {
+                    ATTNW_STAMP(10 + q, j);
 #pragma unroll
 #ifdef ATTN1_X_NOQK
                     for (int k = 0; k < (j == 0 ? D / 16 : 0); ++k) {
@@ -226,6 +249,7 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const uint32_t o_tmem = tmem_base + static_cast<uint32_t>((q * 2 + 1) * kTile);
                 const uint32_t a_base = p_addr + static_cast<uint32_t>(q * L::kPBytes);
                 if (ptx::elect_one()) {
+                    ATTNW_STAMP(12 + q, j);
 #pragma unroll
 #ifdef ATTN1_X_NOPV
                     for (int kk = 0; kk < (j == 0 ? kTile / 16 : 0); ++kk) {
@@ -249,78 +273,116 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (ok && ptx::elect_one()) ptx::umma_commit(&bars->o_full);
         __syncwarp();
     } else if (warp < kSmWarps) {
-        // ================= Softmax warps: one thread per query row =================
-        const int q = warp >> 2;
+        // ================= Softmax warps: two threads per query row, 64 key columns of a tile each =================
+        const int q = warp >> 3;
+        const int half = (warp >> 2) & 1;
         const int quarter = warp & 3;
         if (tile_active[q]) {
             const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(q * 2 * kTile);
-            const uint32_t o_lane = t_lane + static_cast<uint32_t>(kTile);
+            const uint32_t t_own = t_lane + static_cast<uint32_t>(half * kHalf);
+            const uint32_t t_other = t_lane + static_cast<uint32_t>((half ^ 1) * kHalf);
+            const uint32_t o_own = t_lane + static_cast<uint32_t>(kTile + half * (D / 2));  // this thread's D/2 columns of O
             const float c2 = scale_log2e;
             const uint64_t c2c2 = ptx::pack2(c2, c2);
-            // this row of the P tile: 128 bytes in each of the two atoms (64 keys each), 16-byte pieces XOR-swizzled
-            const uint32_t p_row = ptx::smem_u32(smem + L::kPOff + q * L::kPBytes) + static_cast<uint32_t>((quarter * 32 + lane) * 128);
+            // this row in the P tile's atom of this column half (64 keys = 128 bytes, 16-byte pieces XOR-swizzled)
+            const int row = quarter * 32 + lane;
+            const uint32_t p_tile = ptx::smem_u32(smem + L::kPOff + q * L::kPBytes);
+            const uint32_t p_row = p_tile + static_cast<uint32_t>(half * L::kAtomBytes + row * 128);
             const uint32_t sw = static_cast<uint32_t>(lane & 7);
-            float smax = -3.0e38f;  // running maximum of the raw scores of this row
+            float smax = -3.0e38f;  // running maximum of the raw scores of this row (all columns: both threads of a row
+                                    // compute it, each from the whole tile, so they agree without an exchange)
             float mb = -3.0e38f;    // the offset the weights, l and O's row are relative to (follows smax * c2 lazily)
-            float l = 0.0f;
+            float l = 0.0f;         // sum of this thread's weights
             bool ok = true;
 
             for (int j = 0; ok && j < T; ++j) {
                 ok = __all_sync(0xffffffffu, fused_wait(&bars->s_full[q], static_cast<uint32_t>(j) & 1u, abort_flag, kSiteSFull));
                 if (!ok) break;
+                if (quarter == 0 && half == 0 && lane == 0) ATTNW_STAMP(q * 5 + 0, j);
                 ptx::tc_fence_after_sync();
-                // ---- the whole row of scores into registers; the buffer goes back to the MMA issuer at once ----
-                float s[kTile];
+                const int valid = N - j * kTile;  // key columns of this tile that exist
+                // ---- maximum of the other thread's 64 columns (read and dropped) ----
+                float mo = -3.0e38f;
 #pragma unroll
-                for (int c = 0; c < kTile / kChunk; ++c) {
+                for (int c = 0; c < kHalf / kChunk; ++c) {
                     uint32_t r[kChunk];
-                    ptx::tmem_ld_32x32b_x32(t_lane + static_cast<uint32_t>(c * kChunk), r);
+                    ptx::tmem_ld_32x32b_x32(t_other + static_cast<uint32_t>(c * kChunk), r);
+                    ptx::tmem_wait_ld();
+                    if (valid < kTile) {
+#pragma unroll
+                        for (int i = 0; i < kChunk; ++i)
+                            if ((half ^ 1) * kHalf + c * kChunk + i >= valid) r[i] = __float_as_uint(-3.0e38f);
+                    }
+                    float m0 = __uint_as_float(r[0]), m1 = __uint_as_float(r[1]), m2 = __uint_as_float(r[2]), m3 = __uint_as_float(r[3]);
+#pragma unroll
+                    for (int i = 4; i < kChunk; i += 8) {
+                        m0 = ptx::max3(m0, __uint_as_float(r[i + 0]), __uint_as_float(r[i + 1]));
+                        m1 = ptx::max3(m1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                        if (i + 4 < kChunk) {
+                            m2 = ptx::max3(m2, __uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+                            m3 = ptx::max3(m3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
+                        }
+                    }
+                    mo = fmaxf(mo, ptx::max3(fmaxf(m0, m1), m2, m3));
+                }
+                // ---- this thread's 64 scores into registers; the buffer goes back to the MMA issuer at once ----
+                float s[kHalf];
+                {
+                    uint32_t r0[kChunk], r1[kChunk];
+                    ptx::tmem_ld_32x32b_x32(t_own, r0);
+                    ptx::tmem_ld_32x32b_x32(t_own + kChunk, r1);
                     ptx::tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < kChunk; ++i) s[c * kChunk + i] = __uint_as_float(r[i]);
+                    for (int i = 0; i < kChunk; ++i) {
+                        s[i] = __uint_as_float(r0[i]);
+                        s[kChunk + i] = __uint_as_float(r1[i]);
+                    }
                 }
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&bars->s_free[q]);
-                const int valid = N - j * kTile;  // key columns of this tile that exist
+                if (quarter == 0 && half == 0 && lane == 0) ATTNW_STAMP(q * 5 + 1, j);
                 if (valid < kTile) {
 #pragma unroll
-                    for (int i = 0; i < kTile; ++i)
-                        if (i >= valid) s[i] = -3.0e38f;
+                    for (int i = 0; i < kHalf; ++i)
+                        if (half * kHalf + i >= valid) s[i] = -3.0e38f;
                 }
                 // ---- row maximum, lazy offset ----
                 float m0 = s[0], m1 = s[1], m2 = s[2], m3 = s[3];
 #pragma unroll
-                for (int i = 4; i < kTile; i += 8) {
+                for (int i = 4; i < kHalf; i += 8) {
                     m0 = ptx::max3(m0, s[i + 0], s[i + 1]);
                     m1 = ptx::max3(m1, s[i + 2], s[i + 3]);
-                    if (i + 4 < kTile) {
+                    if (i + 4 < kHalf) {
                         m2 = ptx::max3(m2, s[i + 4], s[i + 5]);
                         m3 = ptx::max3(m3, s[i + 6], s[i + 7]);
                     }
                 }
-                smax = fmaxf(smax, ptx::max3(fmaxf(m0, m1), m2, m3));
+                smax = ptx::max3(smax, mo, ptx::max3(fmaxf(m0, m1), m2, m3));
                 const float mb_cand = fmaxf(smax * c2, -3.0e38f);
                 const bool move = j == 0 || mb_cand - mb > kLazy;
+                if (quarter == 0 && half == 0 && lane == 0) ATTNW_STAMP(q * 5 + 2, j);
                 // the P tile and O are free once the MMAs of the previous key tile are complete
-                ok = __all_sync(0xffffffffu, fused_wait(&bars->p_free[q], (static_cast<uint32_t>(j) & 1u) ^ 1u, abort_flag, kSitePFree));
+                ok = __all_sync(0xffffffffu, wait_in_place(&bars->p_free[q], (static_cast<uint32_t>(j) & 1u) ^ 1u, abort_flag, kSitePFree));
                 if (!ok) break;
+                if (quarter == 0 && half == 0 && lane == 0) ATTNW_STAMP(q * 5 + 3, j);
                 if (j == 0) {
                     mb = mb_cand;
                 } else if (__any_sync(0xffffffffu, move)) {
-                    // rescale O's row and l to the new offset (factor 1 for the rows of the warp that do not move)
+                    // rescale this thread's part of O's row and l to the new offset (factor 1 for the rows of the warp
+                    // that do not move; the other thread of the row takes the same decision)
                     const float alpha = move ? ptx::ex2_approx(mb - mb_cand) : 1.0f;
                     if (move) mb = mb_cand;
                     l *= alpha;
                     ptx::tc_fence_after_sync();
 #pragma unroll 1
-                    for (int c = 0; c < D / kChunk; ++c) {
-                        uint32_t r[kChunk];
-                        ptx::tmem_ld_32x32b_x32(o_lane + static_cast<uint32_t>(c * kChunk), r);
+                    for (int c = 0; c < D / 2; c += 8) {  // 8 columns at a time: the row of scores stays in registers
+                        uint32_t r[8];
+                        ptx::tmem_ld_32x32b_x8(o_own + static_cast<uint32_t>(c), r);
                         ptx::tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < kChunk; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                        ptx::tmem_st_32x32b_x32(o_lane + static_cast<uint32_t>(c * kChunk), r);
+                        for (int i = 0; i < 8; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                        ptx::tmem_st_32x32b_x8(o_own + static_cast<uint32_t>(c), r);
                     }
                     ptx::tmem_wait_st();
                 }
@@ -328,7 +390,7 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const uint64_t nmb2 = ptx::pack2(-mb, -mb);
                 uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
-                for (int g = 0; g < kTile / 8; ++g) {  // 8 keys = one 16-byte piece of the row
+                for (int g = 0; g < kHalf / 8; ++g) {  // 8 keys = one 16-byte piece of the row
                     float p[8];
 #pragma unroll
                     for (int i = 0; i < 8; i += 2) {
@@ -341,14 +403,13 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         p[i + 1] = ptx::ex2_approx(x1);
 #endif
                         if (valid < kTile) {  // columns beyond N: weight zero
-                            p[i] = (g * 8 + i < valid) ? p[i] : 0.0f;
-                            p[i + 1] = (g * 8 + i + 1 < valid) ? p[i + 1] : 0.0f;
+                            p[i] = (half * kHalf + g * 8 + i < valid) ? p[i] : 0.0f;
+                            p[i + 1] = (half * kHalf + g * 8 + i + 1 < valid) ? p[i + 1] : 0.0f;
                         }
                         acc[(i >> 1) & 3] = ptx::add2(acc[(i >> 1) & 3], ptx::pack2(p[i], p[i + 1]));
                     }
-                    ptx::st_shared_v4(p_row + static_cast<uint32_t>((g >> 3) * L::kAtomBytes) + ((static_cast<uint32_t>(g & 7) ^ sw) << 4),
-                                      ptx::pack_bf16x2(p[0], p[1]), ptx::pack_bf16x2(p[2], p[3]), ptx::pack_bf16x2(p[4], p[5]),
-                                      ptx::pack_bf16x2(p[6], p[7]));
+                    ptx::st_shared_v4(p_row + ((static_cast<uint32_t>(g) ^ sw) << 4), ptx::pack_bf16x2(p[0], p[1]),
+                                      ptx::pack_bf16x2(p[2], p[3]), ptx::pack_bf16x2(p[4], p[5]), ptx::pack_bf16x2(p[6], p[7]));
                 }
                 float a0, a1, a2, a3;
                 ptx::unpack2(ptx::add2(acc[0], acc[1]), a0, a1);
@@ -358,21 +419,33 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&bars->p_full[q]);
+                if (quarter == 0 && half == 0 && lane == 0) ATTNW_STAMP(q * 5 + 4, j);
             }
 
             // ---- epilogue: O / l -> bf16 -> the P tile's shared memory -> TMA stores ----
             if (ok) ok = __all_sync(0xffffffffu, fused_wait(&bars->o_full, 0, abort_flag, kSiteOFull));
             if (ok) {
+                // every MMA is complete: the K / V ring is free and carries the two partial row sums to each other
+                float* lx = reinterpret_cast<float*>(smem + L::kKOff);
+                lx[(q * 2 + half) * kTile + row] = l;
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&bars->l_full[q]);
+                ok = __all_sync(0xffffffffu, fused_wait(&bars->l_full[q], 0, abort_flag, kSiteLFull));
+            }
+            if (ok) {
+                const float* lx = reinterpret_cast<const float*>(smem + L::kKOff);
+                const float inv_l = 1.0f / (l + lx[(q * 2 + (half ^ 1)) * kTile + row]);
                 ptx::tc_fence_after_sync();
-                const float inv_l = 1.0f / l;
 #pragma unroll 1
-                for (int c = 0; c < D / kChunk; ++c) {
+                for (int c = 0; c < D / 2 / kChunk; ++c) {
                     float o[kChunk];
-                    load_chunk(o_lane + static_cast<uint32_t>(c * kChunk), o);
+                    load_chunk(o_own + static_cast<uint32_t>(c * kChunk), o);
+                    const int col = half * (D / 2) + c * kChunk;  // first of these 32 columns of O
+                    const uint32_t dst = p_tile + static_cast<uint32_t>((col >> 6) * L::kAtomBytes + row * 128);
+                    const uint32_t piece0 = static_cast<uint32_t>((col & 63) >> 3);
 #pragma unroll
                     for (int g = 0; g < 4; ++g)
-                        ptx::st_shared_v4(p_row + static_cast<uint32_t>((c >> 1) * L::kAtomBytes) +
-                                              ((static_cast<uint32_t>((c & 1) * 4 + g) ^ sw) << 4),
+                        ptx::st_shared_v4(dst + (((piece0 + static_cast<uint32_t>(g)) ^ sw) << 4),
                                           ptx::pack_bf16x2(o[g * 8 + 0] * inv_l, o[g * 8 + 1] * inv_l),
                                           ptx::pack_bf16x2(o[g * 8 + 2] * inv_l, o[g * 8 + 3] * inv_l),
                                           ptx::pack_bf16x2(o[g * 8 + 4] * inv_l, o[g * 8 + 5] * inv_l),
@@ -380,12 +453,11 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
-                if (quarter == 0) {
+                if (quarter == 0 && half == 0) {
                     ok = __all_sync(0xffffffffu, fused_wait(&bars->out_filled[q], 0, abort_flag, kSiteOutFilled));
                     if (ok && lane == 0) {
-                        const uint32_t obuf = ptx::smem_u32(smem + L::kPOff + q * L::kPBytes);
                         for (int a = 0; a < L::kAtoms; ++a)
-                            ptx::tma_store_3d(&tm_o, obuf + static_cast<uint32_t>(a * L::kAtomBytes), a * 64, row0 + q * kTile, bh,
+                            ptx::tma_store_3d(&tm_o, p_tile + static_cast<uint32_t>(a * L::kAtomBytes), a * 64, row0 + q * kTile, bh,
                                               ptx::policy_evict_first());
                         ptx::bulk_commit_group();
                         ptx::bulk_wait_group<0>();
