@@ -211,13 +211,8 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(q * 2 * kTile);
                 const uint32_t a_addr = q_addr + static_cast<uint32_t>(q * L::kTileBytes);
                 if (ptx::elect_one()) {
-                    ATTNW_STAMP(10 + q, j);
 #pragma unroll
-#ifdef ATTN1_X_NOQK
-                    for (int k = 0; k < (j == 0 ? D / 16 : 0); ++k) {
-#else
                     for (int k = 0; k < D / 16; ++k) {
-#endif
                         const uint32_t off = static_cast<uint32_t>((k >> 2) * L::kAtomBytes + (k & 3) * 32);
                         ptx::umma_f16_ss(d_tmem, ptx::umma_desc_kmajor_sw128(a_addr + off),
                                          ptx::umma_desc_kmajor_sw128(b_addr + off), idesc_s, k > 0 ? 1u : 0u);
@@ -249,13 +244,8 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const uint32_t o_tmem = tmem_base + static_cast<uint32_t>((q * 2 + 1) * kTile);
                 const uint32_t a_base = p_addr + static_cast<uint32_t>(q * L::kPBytes);
                 if (ptx::elect_one()) {
-                    ATTNW_STAMP(12 + q, j);
 #pragma unroll
-#ifdef ATTN1_X_NOPV
-                    for (int kk = 0; kk < (j == 0 ? kTile / 16 : 0); ++kk) {
-#else
                     for (int kk = 0; kk < kTile / 16; ++kk) {  // 16 keys per instruction
-#endif
                         const uint32_t a_off = static_cast<uint32_t>((kk >> 2) * L::kAtomBytes + (kk & 3) * 32);
                         ptx::umma_f16_ss(o_tmem, ptx::umma_desc_kmajor_sw128(a_base + a_off),
                                          av::umma_desc_mnmajor_sw128(v_addr + static_cast<uint32_t>(kk * 16 * 128), L::kAtomBytes),
@@ -298,7 +288,6 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             for (int j = 0; ok && j < T; ++j) {
                 ok = __all_sync(0xffffffffu, fused_wait(&bars->s_full[q], static_cast<uint32_t>(j) & 1u, abort_flag, kSiteSFull));
                 if (!ok) break;
-                if (quarter == 0 && half == 0 && lane == 0) ATTNW_STAMP(q * 5 + 0, j);
                 ptx::tc_fence_after_sync();
                 const int valid = N - j * kTile;  // key columns of this tile that exist
                 // ---- maximum of the other thread's 64 columns (read and dropped) ----
@@ -341,7 +330,6 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&bars->s_free[q]);
-                if (quarter == 0 && half == 0 && lane == 0) ATTNW_STAMP(q * 5 + 1, j);
                 if (valid < kTile) {
 #pragma unroll
                     for (int i = 0; i < kHalf; ++i)
@@ -361,11 +349,9 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 smax = ptx::max3(smax, mo, ptx::max3(fmaxf(m0, m1), m2, m3));
                 const float mb_cand = fmaxf(smax * c2, -3.0e38f);
                 const bool move = j == 0 || mb_cand - mb > kLazy;
-                if (quarter == 0 && half == 0 && lane == 0) ATTNW_STAMP(q * 5 + 2, j);
                 // the P tile and O are free once the MMAs of the previous key tile are complete
                 ok = __all_sync(0xffffffffu, wait_in_place(&bars->p_free[q], (static_cast<uint32_t>(j) & 1u) ^ 1u, abort_flag, kSitePFree));
                 if (!ok) break;
-                if (quarter == 0 && half == 0 && lane == 0) ATTNW_STAMP(q * 5 + 3, j);
                 if (j == 0) {
                     mb = mb_cand;
                 } else if (__any_sync(0xffffffffu, move)) {
@@ -396,12 +382,8 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     for (int i = 0; i < 8; i += 2) {
                         float x0, x1;
                         ptx::unpack2(ptx::fma2(ptx::pack2(s[g * 8 + i], s[g * 8 + i + 1]), c2c2, nmb2), x0, x1);
-#ifdef ATTN1_X_NOEXP
-                        p[i] = x0; p[i + 1] = x1;
-#else
                         p[i] = ptx::ex2_approx(x0);
                         p[i + 1] = ptx::ex2_approx(x1);
-#endif
                         if (valid < kTile) {  // columns beyond N: weight zero
                             p[i] = (half * kHalf + g * 8 + i < valid) ? p[i] : 0.0f;
                             p[i + 1] = (half * kHalf + g * 8 + i + 1 < valid) ? p[i + 1] : 0.0f;
@@ -419,7 +401,6 @@ attn_onepass_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&bars->p_full[q]);
-                if (quarter == 0 && half == 0 && lane == 0) ATTNW_STAMP(q * 5 + 4, j);
             }
 
             // ---- epilogue: O / l -> bf16 -> the P tile's shared memory -> TMA stores ----
