@@ -9,6 +9,7 @@ Each function is the definition written out in double precision:
 * :func:`softmax_rows` - Softmax definition of Section VI with the max subtraction of Eq. 1.
 * :func:`attnw` / :func:`attnw_rows` - ``softmax(scale * Q K^T)`` of Section IV (restated for
   ``n x d_k`` inputs and an ``n x n`` output in Section VII).
+* :func:`project` - the linear transformation of the inputs into queries or keys (Section IV), ``X W_h`` per head.
 * :func:`paper_cpu_softmax` - the fp32 single-core CPU program of Section VI-A (caching and
   recomputing forms), a timed context baseline, not the parity oracle.
 
@@ -59,6 +60,8 @@ def _load():
             lib.oracle_attn.argtypes = [vp, vp, vp, vp, c_long, c_long, c_long, c_long, c_float, c_int]
             lib.oracle_attn_rows.argtypes = [vp, vp, vp, vp, c_long, c_long, c_long, c_long, c_float,
                                              vp, c_long, c_int]
+            lib.oracle_project.argtypes = [vp, vp, vp, c_long, c_long, c_long, c_long, c_long, vp, c_long]
+            lib.oracle_project.restype = c_int
             for f in (lib.oracle_softmax_rows, lib.oracle_softmax_rows_subset, lib.oracle_attnw,
                       lib.oracle_attnw_rows, lib.oracle_scores_rows, lib.oracle_attn, lib.oracle_attn_rows):
                 f.restype = c_int
@@ -166,6 +169,27 @@ def attn(Q, K, V, scale: float, row_ids=None, threads: int | None = None) -> np.
     _check(_load().oracle_attn_rows(_ptr(Q), _ptr(K), _ptr(V), _ptr(O), B, H, N, d, float(np.float32(scale)),
                                     _ptr(ids), ids.size, threads or host_cores()), "attn_rows")
     return O
+
+
+def project(X, W, row_ids=None) -> np.ndarray:
+    """Queries (or keys) from the inputs (Section IV): ``out[b,h,n,c] = sum_m X[b,n,m] W[h,c,m]`` for bf16 bit
+    patterns ``X [B,N,d_model]`` and ``W [H,d,d_model]`` (row ``c`` of head ``h`` is column ``c`` of that head's
+    parameter matrix) -> float64 ``[B,H,N,d]``, or ``[len(row_ids), d]`` for the listed global rows
+    ``(b*H + h)*N + n``."""
+    X = _as_bf16_bits(X, "X")
+    W = _as_bf16_bits(W, "W")
+    if X.ndim != 3 or W.ndim != 3 or X.shape[2] != W.shape[2]:
+        raise ValueError("X must be [B,N,d_model] and W [H,d,d_model]")
+    B, N, d_model = X.shape
+    H, d, _ = W.shape
+    if row_ids is None:
+        out = np.empty((B, H, N, d), dtype=np.float64)
+        _check(_load().oracle_project(_ptr(X), _ptr(W), _ptr(out), B, N, d_model, H, d, None, 0), "project")
+        return out
+    ids = np.ascontiguousarray(row_ids, dtype=np.int64)
+    out = np.empty((ids.size, d), dtype=np.float64)
+    _check(_load().oracle_project(_ptr(X), _ptr(W), _ptr(out), B, N, d_model, H, d, _ptr(ids), ids.size), "project")
+    return out
 
 
 def scores_rows(Q, K, row_ids) -> np.ndarray:

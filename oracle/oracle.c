@@ -328,3 +328,33 @@ int oracle_scores_rows(const uint16_t *Q, const uint16_t *K, double *S, long B, 
     }
     return 0;
 }
+
+/* ---- the linear transformation of the inputs into queries (or keys), Section IV: per head h,
+ *      Q_h = X W_h, written out as Q[b,h,n,c] = sum_m X[b,n,m] * W[h,c,m], m ascending.
+ *      X: [B, N, d_model] bfloat16 bits.  W: [H, d, d_model] bfloat16 bits (row c of head h holds column c of
+ *      that head's parameter matrix).  Only the listed global rows (b*H + h)*N + n, or all rows when row_ids
+ *      is NULL (then n_ids is ignored); out is rows x d. */
+int oracle_project(const uint16_t *X, const uint16_t *W, double *out, long B, long N, long d_model, long H,
+                   long d, const long *row_ids, long n_ids)
+{
+    if (!X || !W || !out || B < 1 || N < 1 || d_model < 1 || H < 1 || d < 1)
+        return -2;
+    long rows = row_ids ? n_ids : B * H * N;
+    if (rows < 1)
+        return -2;
+    for (long r = 0; r < rows; ++r) {
+        long g = row_ids ? row_ids[r] : r;
+        if (g < 0 || g >= B * H * N)
+            return -3;
+        long n = g % N, h = (g / N) % H, b = g / (N * H);
+        const uint16_t *x = X + ((size_t)b * (size_t)N + (size_t)n) * (size_t)d_model;
+        for (long c = 0; c < d; ++c) {
+            const uint16_t *w = W + ((size_t)h * (size_t)d + (size_t)c) * (size_t)d_model;
+            double s = 0.0;
+            for (long m = 0; m < d_model; ++m)
+                s += bf16_to_double(x[m]) * bf16_to_double(w[m]);
+            out[(size_t)r * (size_t)d + (size_t)c] = s;
+        }
+    }
+    return 0;
+}

@@ -362,3 +362,62 @@ def test_attention_against_float64_library(shape, sigma):
     assert np.max(np.abs(O - ref)) <= 1e-12
     ids = [0, 5, shape[0] * shape[1] * shape[2] - 1]
     assert np.array_equal(oracle.attn(q, k, v, scale, row_ids=ids), O.reshape(-1, shape[3])[ids])
+
+
+# ---- queries and keys from the inputs: the linear transformation of Section IV ----------------
+
+def rand_xw(B, N, d_model, H, d, sigma_w=None, stream=600):
+    x = inputs.normal_bf16_bits(7, stream, B * N * d_model, 1.0).reshape(B, N, d_model)
+    w = inputs.normal_bf16_bits(7, stream + 1, H * d * d_model, sigma_w or d_model ** -0.5).reshape(H, d, d_model)
+    return x, w
+
+
+def test_projection_with_selector_weights_copies_input_columns():
+    # W[h, c, :] = unit vector e_{h*d + c}: head h of the output is columns h*d .. h*d+d-1 of X, exactly.
+    B, N, H, d = 2, 9, 3, 4
+    d_model = H * d + 5
+    x, _ = rand_xw(B, N, d_model, H, d)
+    w = np.zeros((H, d, d_model), dtype=np.float32)
+    for h in range(H):
+        for c in range(d):
+            w[h, c, h * d + c] = 1.0
+    out = oracle.project(x, bits(w))
+    for h in range(H):
+        assert np.array_equal(out[:, h], dec(x)[:, :, h * d:(h + 1) * d])   # catches swapped head / feature axes
+
+
+def test_projection_small_integers_exact_and_brute_force():
+    rng = np.random.default_rng(5)
+    B, N, d_model, H, d = 2, 3, 6, 2, 3
+    xv = rng.integers(-4, 5, size=(B, N, d_model)).astype(np.float32)
+    wv = rng.integers(-4, 5, size=(H, d, d_model)).astype(np.float32)
+    out = oracle.project(bits(xv), bits(wv))
+    for b in range(B):
+        for h in range(H):
+            for n in range(N):
+                for c in range(d):
+                    want = sum(int(xv[b, n, m]) * int(wv[h, c, m]) for m in range(d_model))   # integers: exact
+                    assert out[b, h, n, c] == want
+
+
+def test_projection_is_linear_and_heads_are_independent():
+    x, w = rand_xw(1, 20, 48, 2, 8, stream=610)
+    out = oracle.project(x, w)
+    w2 = dec(w).copy()
+    w2[1] *= 2.0                                   # exact in bf16
+    out2 = oracle.project(x, bits(w2.astype(np.float32)))
+    assert np.array_equal(out2[:, 0], out[:, 0])
+    assert np.array_equal(out2[:, 1], 2.0 * out[:, 1])
+    x0 = dec(x).copy()
+    x0[:, 7] = 0.0                                 # a zero input row gives a zero output row in every head
+    assert np.all(oracle.project(bits(x0.astype(np.float32)), w)[:, :, 7] == 0.0)
+
+
+def test_projection_against_float64_library_and_row_subset():
+    B, N, d_model, H, d = 2, 33, 96, 3, 16
+    x, w = rand_xw(B, N, d_model, H, d, stream=620)
+    out = oracle.project(x, w)
+    ref = np.einsum("bnm,hcm->bhnc", dec(x), dec(w))
+    assert np.max(np.abs(out - ref)) <= 1e-13 * d_model
+    ids = [0, 40, B * H * N - 1]
+    assert np.array_equal(oracle.project(x, w, row_ids=ids), out.reshape(-1, d)[ids])
