@@ -73,6 +73,24 @@ int attn_fused(const void* Q, const void* K, const void* V, void* O, int B, int 
                void* stream);
 
 /*
+ * attnw_project_qk: the linear transformation of the inputs into queries and keys in front of the attention weights
+ * (Section IV; a step the paper leaves to the vendor's matmul and names as future work in Section IX), for all heads in
+ * one launch:   Q[b,h,n,c] = sum_m X[b,n,m] * Wq[h,c,m],   K[b,h,n,c] = sum_m X[b,n,m] * Wk[h,c,m].
+ *
+ *   X        device, bfloat16, [B, N, d_model]                  (read only)
+ *   Wq, Wk   device, bfloat16, [H, d, d_model]: row c of head h holds column c of that head's parameter matrix, i.e.
+ *            the matrices are stored transposed, contiguous along d_model               (read only)
+ *   Q, K     device, bfloat16, [B, H, N, d] - the layout attnw_fused and attn_fused read; every element is written
+ *            exactly once; must not overlap each other or any input
+ *   B,N,H    >= 1 (no divisibility condition);  d in {64, 128};  d_model >= 8, a multiple of 8 (else
+ *            ATTNW_ERR_MISALIGNED), at most 2^20
+ * Products are accumulated in float32 on the tensor cores over d_model in ascending blocks of 16; the results are
+ * rounded to bfloat16 (nearest even).
+ */
+int attnw_project_qk(const void* X, const void* Wq, const void* Wk, void* Q, void* K, int B, int N, int d_model, int H,
+                     int d, void* stream);
+
+/*
  * Which kernel attn_fused uses (process-wide; the results agree within the stated tolerance):
  *   0  default: the one-pass kernel
  *   1  two-pass kernel: row maxima and sums in a first pass over the keys, normalised weights times V in a second

@@ -18,6 +18,7 @@ _vp, _int, _ll, _float = ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong, ctype
 # name -> (restype, argtypes); mirrors include/attnw.h one to one
 SIGNATURES = {
     "attn_fused": (_int, [_vp, _vp, _vp, _vp, _int, _int, _int, _int, _float, _vp]),
+    "attnw_project_qk": (_int, [_vp, _vp, _vp, _vp, _vp, _int, _int, _int, _int, _int, _vp]),
     "attnw_fused": (_int, [_vp, _vp, _vp, _int, _int, _int, _int, _float, _vp]),
     "attnw_fused_f32": (_int, [_vp, _vp, _vp, _int, _int, _int, _int, _float, _vp]),
     "softmax_rows": (_int, [_vp, _vp, _ll, _ll, _vp]),
@@ -155,6 +156,32 @@ def attn_fused(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, scale: float, 
         _check(lib.attn_fused(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), B, H, N, d, float(scale),
                               _stream_ptr(stream)), "attn_fused")
     return O
+
+
+def project_qk(X: torch.Tensor, Wq: torch.Tensor, Wk: torch.Tensor, Q: torch.Tensor | None = None,
+               K: torch.Tensor | None = None, stream=None) -> tuple[torch.Tensor, torch.Tensor]:
+    """Queries and keys from the inputs: ``Q[b,h] = X[b] Wq[h]^T``, ``K[b,h] = X[b] Wk[h]^T`` for CUDA bfloat16
+    ``X [B, N, d_model]`` and ``Wq, Wk [H, d, d_model]`` -> ``Q, K [B, H, N, d]`` (bfloat16), the layout
+    ``attnw_fused`` and ``attn_fused`` read.  Asynchronous on ``stream`` (default: torch's current stream)."""
+    for t, name in ((X, "X"), (Wq, "Wq"), (Wk, "Wk")):
+        _require_cuda(t, name, torch.bfloat16)
+    if X.dim() != 3 or Wq.dim() != 3 or Wq.shape != Wk.shape or Wq.shape[2] != X.shape[2]:
+        raise ValueError("X must be [B, N, d_model] and Wq, Wk [H, d, d_model]")
+    B, N, d_model = X.shape
+    H, d, _ = Wq.shape
+    outs = []
+    for t, name in ((Q, "Q"), (K, "K")):
+        if t is None:
+            t = torch.empty((B, H, N, d), dtype=torch.bfloat16, device=X.device)
+        else:
+            _require_cuda(t, name, torch.bfloat16)
+            if tuple(t.shape) != (B, H, N, d):
+                raise ValueError(f"{name} must be [B, H, N, d]")
+        outs.append(t)
+    with torch.cuda.device(X.device):
+        _check(lib.attnw_project_qk(X.data_ptr(), Wq.data_ptr(), Wk.data_ptr(), outs[0].data_ptr(), outs[1].data_ptr(), B, N,
+                                    d_model, H, d, _stream_ptr(stream)), "attnw_project_qk")
+    return outs[0], outs[1]
 
 
 def softmax_rows(S: torch.Tensor, P: torch.Tensor | None = None, out_dtype: torch.dtype = torch.bfloat16,

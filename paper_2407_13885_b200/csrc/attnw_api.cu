@@ -15,6 +15,7 @@
 #include "attnw_fused.cuh"
 #include "attn_fused.cuh"
 #include "attn_onepass.cuh"
+#include "project_qk.cuh"
 #include "attnw_resident.cuh"
 #include "softmax_rows.cuh"
 
@@ -362,6 +363,55 @@ int validate_attn(const void* Q, const void* K, const void* V, const void* O, in
     return ATTNW_OK;
 }
 
+// Host-only checks of the projection call; no CUDA call is made here.
+int validate_project(const void* X, const void* Wq, const void* Wk, const void* Q, const void* K, int B, int N, int d_model,
+                     int H, int d) {
+    if (!X || !Wq || !Wk || !Q || !K) return ATTNW_ERR_NULL_POINTER;
+    if (B < 1 || N < 1 || d_model < 1 || H < 1 || d < 1) return ATTNW_ERR_BAD_SHAPE;
+    if (N > (1 << 24) || d_model > (1 << 20)) return ATTNW_ERR_BAD_SHAPE;  // keeps every tensor-map stride below 2^40 bytes
+    const long long bh = static_cast<long long>(B) * H;
+    if (bh > INT_MAX || static_cast<long long>(H) * d > INT_MAX) return ATTNW_ERR_BAD_SHAPE;
+    const long long col_tiles = (static_cast<long long>(H) * d + proj::kCols - 1) / proj::kCols;
+    const long long row_tiles = (static_cast<long long>(N) + proj::kRows - 1) / proj::kRows;
+    if (2 * col_tiles * row_tiles * B > INT_MAX) return ATTNW_ERR_BAD_SHAPE;
+    if (d != 64 && d != 128) return ATTNW_ERR_UNSUPPORTED;
+    if (d_model % 8 != 0) return ATTNW_ERR_MISALIGNED;  // rows of X and of the weights must start on 16-byte boundaries
+    if (!aligned16(X) || !aligned16(Wq) || !aligned16(Wk) || !aligned16(Q) || !aligned16(K)) return ATTNW_ERR_MISALIGNED;
+    const unsigned long long x_bytes = static_cast<unsigned long long>(B) * N * d_model * 2ull;
+    const unsigned long long w_bytes = static_cast<unsigned long long>(H) * d * d_model * 2ull;
+    const unsigned long long o_bytes = static_cast<unsigned long long>(bh) * N * d * 2ull;
+    if (overlaps(Q, o_bytes, K, o_bytes)) return ATTNW_ERR_ALIASING;
+    for (const void* out : {Q, K})
+        if (overlaps(out, o_bytes, X, x_bytes) || overlaps(out, o_bytes, Wq, w_bytes) || overlaps(out, o_bytes, Wk, w_bytes))
+            return ATTNW_ERR_ALIASING;
+    return ATTNW_OK;
+}
+
+int launch_project(const void* X, const void* Wq, const void* Wk, void* Q, void* K, int B, int N, int d_model, int H, int d,
+                   cudaStream_t stream) {
+    CUtensorMap tm_x, tm_wq, tm_wk, tm_q, tm_k;
+    const uint64_t hd = static_cast<uint64_t>(H) * d;
+    int rc = encode_3d(&tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, X, d_model, N, B, proj::kKSlice, 128);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_wq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Wq, d_model, hd, 1, proj::kKSlice, 128);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_wk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Wk, d_model, hd, 1, proj::kKSlice, 128);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Q, d, N, static_cast<uint64_t>(B) * H, 64, 128);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, K, d, N, static_cast<uint64_t>(B) * H, 64, 128);
+    if (rc != ATTNW_OK) return rc;
+    if (cudaFuncSetAttribute(proj::project_qk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, proj::kDynamicBytes) !=
+        cudaSuccess) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    const int col_tiles = static_cast<int>((hd + proj::kCols - 1) / proj::kCols);
+    const int row_tiles = (N + proj::kRows - 1) / proj::kRows;
+    const unsigned ctas = static_cast<unsigned>(2 * col_tiles) * static_cast<unsigned>(row_tiles) * static_cast<unsigned>(B);
+    proj::project_qk_kernel<<<ctas, proj::kThreads, proj::kDynamicBytes, stream>>>(tm_x, tm_wq, tm_wk, tm_q, tm_k, N, d_model, H,
+                                                                                     d, col_tiles, row_tiles);
+    if (cudaGetLastError() != cudaSuccess) return ATTNW_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTNW_OK;
+}
+
 template <typename OutT>
 int fused_entry(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream) {
     int rc = validate_fused(Q, K, P, B, H, N, d, scale, sizeof(OutT));
@@ -539,6 +589,18 @@ int attn_fused(const void* Q, const void* K, const void* V, void* O, int B, int 
         return d == 64 ? launch_attn<64>(Q, K, V, O, B * H, N, scale, s) : launch_attn<128>(Q, K, V, O, B * H, N, scale, s);
     return d == 64 ? launch_attn_onepass<64>(Q, K, V, O, B * H, N, scale, s)
                    : launch_attn_onepass<128>(Q, K, V, O, B * H, N, scale, s);
+}
+
+int attnw_project_qk(const void* X, const void* Wq, const void* Wk, void* Q, void* K, int B, int N, int d_model, int H, int d,
+                     void* stream) {
+    int rc = validate_project(X, Wq, Wk, Q, K, B, N, d_model, H, d);
+    if (rc != ATTNW_OK) return rc;
+    DeviceInfo* dev = nullptr;
+    rc = current_device(&dev);
+    if (rc != ATTNW_OK) return rc;
+    rc = load_encoder();
+    if (rc != ATTNW_OK) return rc;
+    return launch_project(X, Wq, Wk, Q, K, B, N, d_model, H, d, static_cast<cudaStream_t>(stream));
 }
 
 int attnw_set_attn_variant(int variant) {

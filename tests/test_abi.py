@@ -76,6 +76,27 @@ def test_fused_argument_errors_are_host_side(lib):
     assert f(A, A, 0x900000, 65536, 65536, 128, 64, 0.125, None) == 2  # B*H overflows
 
 
+def test_projection_argument_errors_are_host_side(lib):
+    f = lib.attnw_project_qk
+    X, WQ, WK, Q, K = 0x100000, 0x2000000, 0x3000000, 0x4000000, 0x5000000
+    for i in range(5):
+        ptrs = [X, WQ, WK, Q, K]
+        ptrs[i] = None
+        assert f(*ptrs, 1, 128, 64, 1, 64, None) == 1
+    assert f(X, WQ, WK, Q, K, 0, 128, 64, 1, 64, None) == 2
+    assert f(X, WQ, WK, Q, K, 1, 0, 64, 1, 64, None) == 2
+    assert f(X, WQ, WK, Q, K, 1, 128, 0, 1, 64, None) == 2
+    assert f(X, WQ, WK, Q, K, 1, 128, 64, 0, 64, None) == 2
+    assert f(X, WQ, WK, Q, K, 1, 128, (1 << 20) + 8, 1, 64, None) == 2
+    assert f(X, WQ, WK, Q, K, 1, 128, 64, 1, 32, None) == 4            # d must be 64 or 128
+    assert f(X, WQ, WK, Q, K, 1, 128, 68, 1, 64, None) == 3            # rows of X would not start on 16 bytes
+    assert f(X + 2, WQ, WK, Q, K, 1, 128, 64, 1, 64, None) == 3
+    assert f(X, WQ, WK, Q, K + 8, 1, 128, 64, 1, 64, None) == 3
+    assert f(X, WQ, WK, Q, Q, 1, 128, 64, 1, 64, None) == 7            # Q and K may not share memory
+    assert f(X, WQ, WK, X, K, 1, 128, 64, 1, 64, None) == 7            # an output over an input
+    assert f(X, WQ, WK, Q, WK + 16, 1, 128, 64, 1, 64, None) == 7
+
+
 def test_rows_argument_errors_are_host_side(lib):
     f = lib.softmax_rows
     assert f(None, A, 4, 8, None) == 1
