@@ -265,6 +265,36 @@ def attention_config(binding, inputs, name, peaks, steps=20, warmup=3):
             "peak_tflops": peaks["bf16_tflops"], "algorithmic_flops": flops, "steps": steps}
 
 
+def projection_inputs(inputs, w, B):
+    """X [B, N, d_model] ~ N(0, 1) and Wq, Wk [H, d, d_model] ~ N(0, 1/d_model) with d_model = H * d: the inputs that
+    produce queries and keys distributed like the headline workload's (bf16 bit patterns, seeded, on their own streams)."""
+    dm = w.H * w.d
+    x = inputs.normal_bf16_bits(inputs.SEED, 2 * w.cfg_id + 200, B * w.N * dm, 1.0)
+    wq = inputs.normal_bf16_bits(inputs.SEED, 2 * w.cfg_id + 201, w.H * w.d * dm, dm ** -0.5)
+    wk = inputs.normal_bf16_bits(inputs.SEED, 2 * w.cfg_id + 202, w.H * w.d * dm, dm ** -0.5)
+    return x, wq, wk, dm
+
+
+def projection_config(binding, inputs, name, peaks, steps=20, warmup=3):
+    """Short kernel-only measurement of attnw_project_qk (queries and keys from the inputs, Section IV) for the shape of
+    one of the configurations with d_model = H * d (reported beside the headline, not part of it)."""
+    import torch
+    w = inputs.WORKLOADS[name]
+    x, wq, wk, dm = projection_inputs(inputs, w, w.B)
+    as_t = lambda a, shape: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).reshape(shape).cuda()  # noqa: E731
+    X, Wq, Wk = as_t(x, (w.B, w.N, dm)), as_t(wq, (w.H, w.d, dm)), as_t(wk, (w.H, w.d, dm))
+    Q = torch.empty((w.B, w.H, w.N, w.d), dtype=torch.bfloat16, device="cuda")
+    K = torch.empty_like(Q)
+    ms = time_launches(lambda: binding.project_qk(X, Wq, Wk, Q=Q, K=K), steps, warmup, torch.cuda.synchronize) / steps
+    flops = 2.0 * w.B * w.N * dm * 2 * w.H * w.d      # two products of [B N, d_model] with [d_model, H d]
+    bytes_alg = (w.B * w.N * dm + 2 * w.H * w.d * dm + 2 * w.B * w.H * w.N * w.d) * 2
+    t_flop = flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = bytes_alg / (peaks["hbm_gbs"] * 1e9)
+    return {"op": f"attnw_project_qk: Q, K = X Wq, X Wk, bf16, d_model={dm}", "ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+            "roofline_frac": max(t_hbm, t_flop) / (ms * 1e-3), "bound": "tensor" if t_flop >= t_hbm else "hbm",
+            "peak_tflops": peaks["bf16_tflops"], "algorithmic_flops": flops, "steps": steps}
+
+
 def run_profile_case(args):
     """A reduced case of one kernel for profiler captures (`--profile fused|rows`): the same kernel and
     tile configuration as the headline launch on inputs that still exceed the L2 but hold well under a
@@ -296,6 +326,15 @@ def run_profile_case(args):
         O = torch.empty_like(Q)
         fn = lambda: binding.attn_fused(Q, K, V, w.scale, O=O)  # noqa: E731
         desc = f"attn_fused B=1 H={heads} N={w.N} d={w.d}"
+    elif args.profile == "project":
+        w = inputs.WORKLOADS[args.workload]
+        x, wq, wk, dm = projection_inputs(inputs, w, 1)   # one batch entry of the configuration
+        as_t = lambda a, shape: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).reshape(shape).cuda()  # noqa: E731
+        X, Wq, Wk = as_t(x, (1, w.N, dm)), as_t(wq, (w.H, w.d, dm)), as_t(wk, (w.H, w.d, dm))
+        Q = torch.empty((1, w.H, w.N, w.d), dtype=torch.bfloat16, device="cuda")
+        K = torch.empty_like(Q)
+        fn = lambda: binding.project_qk(X, Wq, Wk, Q=Q, K=K)  # noqa: E731
+        desc = f"attnw_project_qk B=1 N={w.N} d_model={dm} H={w.H} d={w.d}"
     else:
         base = inputs.WORKLOADS["c4"]
         rows = 8192
@@ -461,6 +500,8 @@ def run_ours(args):
             torch.cuda.empty_cache()
         other["attention_c3"] = attention_config(binding, inputs, "c3", peaks)
         torch.cuda.empty_cache()
+        other["project_qk_c3"] = projection_config(binding, inputs, "c3", peaks)
+        torch.cuda.empty_cache()
         line["other_configs"] = other
     print(json.dumps(line))
     return 0
@@ -482,7 +523,7 @@ def main():
     ap.add_argument("--sustained-seconds", type=float, default=2.0)
     ap.add_argument("--variant", choices=["auto", "two_pass", "resident"], default="auto",
                     help="kernel behind attnw_fused (see attnw_set_fused_variant)")
-    ap.add_argument("--profile", choices=["fused", "rows", "attention"], default=None,
+    ap.add_argument("--profile", choices=["fused", "rows", "attention", "project"], default=None,
                     help="run a reduced case of one kernel for an ncu capture instead of the benchmark")
     args = ap.parse_args()
     if args.impl == "reference":

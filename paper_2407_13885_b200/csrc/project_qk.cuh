@@ -18,6 +18,7 @@ constexpr int kRows = 256;        // rows of X per CTA (two MMA row blocks)
 constexpr int kCols = 256;        // output features per CTA
 constexpr int kKSlice = 64;       // d_model elements per stage: one 128-byte swizzle atom
 constexpr int kStages = 3;
+constexpr int kGroupCols = 16;    // column tiles walked together (32 MB of weights at d_model = 4096)
 constexpr int kEpiWarps = 8;      // TMEM lane quarter (4) x column half (2)
 constexpr int kProducer = 8;
 constexpr int kMma = 9;
@@ -45,8 +46,9 @@ struct Barriers {
 };
 static_assert(sizeof(Barriers) <= 256, "barrier block must fit its slot");
 
-// grid: 2 * col_tiles * B * row_tiles CTAs; the 2 * col_tiles tiles (Q's, then K's) of one block of rows are neighbours,
-// so that block of X is read from HBM once and the weights stay in L2
+// grid: 2 * col_tiles * B * row_tiles CTAs.  The column tiles (Q's, then K's) are walked in groups of kGroupCols: within
+// a group the tiles of one block of rows are neighbours (that block of X is fetched once per group) and the group's
+// slice of the weights (kGroupCols x 256 x d_model) is small enough to stay in L2 while all row blocks pass.
 __global__ void __launch_bounds__(kThreads, 1)
 project_qk_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_wq,
                   const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_q,
@@ -62,8 +64,13 @@ project_qk_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int tile_x = static_cast<int>(blockIdx.x % static_cast<unsigned>(2 * col_tiles));
-    const int tile_y = static_cast<int>(blockIdx.x / static_cast<unsigned>(2 * col_tiles));
+    const int n_x = 2 * col_tiles, n_y = static_cast<int>(gridDim.x) / n_x;
+    const int n_groups = (n_x + kGroupCols - 1) / kGroupCols;
+    const int group = min(static_cast<int>(blockIdx.x) / (kGroupCols * n_y), n_groups - 1);
+    const int in_group = static_cast<int>(blockIdx.x) - group * kGroupCols * n_y;
+    const int width = group == n_groups - 1 ? n_x - group * kGroupCols : kGroupCols;
+    const int tile_x = group * kGroupCols + in_group % width;
+    const int tile_y = in_group / width;
     const bool keys = tile_x >= col_tiles;  // this CTA computes a tile of K, not of Q
     const int c0 = (tile_x - (keys ? col_tiles : 0)) * kCols;  // first output feature (of H * d)
     const int b = tile_y / row_tiles;
