@@ -218,8 +218,9 @@ def time_launches(fn, steps, warmup, stream_sync):
     return start.elapsed_time(stop)
 
 
-def secondary_config(binding, inputs, name, peaks, steps=20, warmup=3):
-    """Short kernel-only measurement of one of the other configurations (reported, not the headline)."""
+def secondary_config(binding, inputs, name, peaks, steps=20, warmup=3, rows_variant="auto"):
+    """Short kernel-only measurement of one of the other configurations (reported, not the headline).
+    ``rows_variant``: the form of softmax_rows (Section VI-A's caching / recomputing comparison)."""
     import torch
     w = inputs.WORKLOADS[name]
     if w.kind == "rows":
@@ -236,7 +237,11 @@ def secondary_config(binding, inputs, name, peaks, steps=20, warmup=3):
         P = torch.empty((w.B, w.H, w.N, w.N), dtype=torch.bfloat16 if w.p_dtype == "bf16" else torch.float32,
                         device="cuda")
         fn = lambda: binding.attnw_fused(Q, K, w.scale, P=P)  # noqa: E731
-    ms = time_launches(fn, steps, warmup, torch.cuda.synchronize) / steps
+    binding.set_rows_variant(rows_variant)
+    try:
+        ms = time_launches(fn, steps, warmup, torch.cuda.synchronize) / steps
+    finally:
+        binding.set_rows_variant("auto")
     bytes_alg = w.in_bytes + w.p_bytes
     t_hbm = bytes_alg / (peaks["hbm_gbs"] * 1e9)
     t_flop = w.flops / (peaks["bf16_tflops"] * 1e12)
@@ -498,6 +503,8 @@ def run_ours(args):
         for name in ("c4", "c5", "c2"):
             other[name] = secondary_config(binding, inputs, name, peaks)
             torch.cuda.empty_cache()
+        other["c4_recomputing"] = secondary_config(binding, inputs, "c4", peaks, rows_variant="recomputing")
+        torch.cuda.empty_cache()
         other["attention_c3"] = attention_config(binding, inputs, "c3", peaks)
         torch.cuda.empty_cache()
         other["project_qk_c3"] = projection_config(binding, inputs, "c3", peaks)

@@ -136,6 +136,17 @@ int softmax_rows(const void* S, void* P, long long rows, long long cols, void* s
 int softmax_rows_f32(const void* S, void* P, long long rows, long long cols, void* stream);
 
 /*
+ * Which form of the row Softmax softmax_rows uses (process-wide; Section VI-A compares the two on its hardware):
+ *   0  by row length (default): rows of up to 32768 columns are read once and kept in registers ("caching", one
+ *      exponential per element); longer rows are read twice and their exponentials recomputed
+ *   1  caching only: a call with cols > 32768 returns ATTNW_ERR_UNSUPPORTED
+ *   2  recomputing for every row length: first read for the running maximum and sum, second read (mostly from L2)
+ *      recomputes the exponentials - two exponentials and two reads per element, nothing kept on chip
+ * Returns ATTNW_ERR_BAD_SHAPE for any other value.
+ */
+int attnw_set_rows_variant(int variant);
+
+/*
  * The same two operations for callers whose data lives in HOST memory (Section III describes
  * the host program's write-buffer / run / read-buffer sequence).  Pointers are HOST pointers
  * (pinned memory gives the fastest copies; pageable memory works).  The call copies the

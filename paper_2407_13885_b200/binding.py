@@ -29,6 +29,7 @@ SIGNATURES = {
     "attnw_query_status": (_int, [_vp, ctypes.POINTER(ctypes.c_uint)]),
     "attnw_set_fused_variant": (_int, [_int]),
     "attnw_set_attn_variant": (_int, [_int]),
+    "attnw_set_rows_variant": (_int, [_int]),
     "attnw_launch_count": (_ll, [_int]),
     "attnw_strerror": (ctypes.c_char_p, [_int]),
     "attnw_version": (_int, []),
@@ -78,6 +79,15 @@ def set_fused_variant(variant: str | int) -> None:
     (the resident kernel with the reduce-and-broadcast exchange)."""
     code = FUSED_VARIANTS[variant] if isinstance(variant, str) else int(variant)
     _check(lib.attnw_set_fused_variant(code), "attnw_set_fused_variant")
+
+
+ROWS_VARIANTS = {"auto": 0, "caching": 1, "recomputing": 2}
+
+
+def set_rows_variant(variant: str | int) -> None:
+    """Selects the form of ``softmax_rows``: "auto" (by row length), "caching" or "recomputing" (Section VI-A)."""
+    code = ROWS_VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    _check(lib.attnw_set_rows_variant(code), "attnw_set_rows_variant")
 
 
 ATTN_VARIANTS = {"auto": 0, "two_pass": 1, "one_pass": 2}

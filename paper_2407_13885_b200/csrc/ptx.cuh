@@ -78,7 +78,7 @@ __device__ __forceinline__ uint64_t policy_evict_last() {
     return p;
 }
 
-// ---- TMA: tiled tensor copies (no multicast anywhere) -------------------------------------
+// ---- TMA: tiled tensor copies (every load is for this CTA alone) --------------------------
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
 }

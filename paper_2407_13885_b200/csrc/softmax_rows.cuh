@@ -188,11 +188,12 @@ inline cudaError_t sr_launch_reg(const float* S, OutT* P, long long rows, int co
 
 constexpr long long kSoftmaxRowsRegTierMaxCols = 32768;
 
+// recomputing: take the streaming tier whatever the row length (the "recomputing" form of Section VI-A on request)
 template <typename OutT>
 inline cudaError_t softmax_rows_launch(const float* S, OutT* P, long long rows, long long cols, int sm_count,
-                                       cudaStream_t stream) {
+                                       cudaStream_t stream, bool recomputing = false) {
     const long long nvec = cols / 4;
-    if (cols > kSoftmaxRowsRegTierMaxCols) {
+    if (recomputing || cols > kSoftmaxRowsRegTierMaxCols) {
         const long long cap = static_cast<long long>(sm_count) * 4;
         const unsigned grid = static_cast<unsigned>(rows < cap ? rows : cap);
         softmax_rows_stream_kernel<OutT><<<grid, 1024, 0, stream>>>(S, P, rows, cols);

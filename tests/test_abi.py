@@ -118,6 +118,13 @@ def test_fused_variant_knob(lib):
         assert lib.attnw_set_fused_variant(v) == 0
 
 
+def test_rows_variant_knob(lib):
+    assert lib.attnw_set_rows_variant(3) == 2
+    assert lib.attnw_set_rows_variant(-1) == 2
+    for v in (1, 2, 0):
+        assert lib.attnw_set_rows_variant(v) == 0
+
+
 def test_attention_variant_knob(lib):
     assert lib.attnw_set_attn_variant(3) == 2
     assert lib.attnw_set_attn_variant(-1) == 2

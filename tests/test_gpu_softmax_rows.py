@@ -34,6 +34,34 @@ def test_rows_match_oracle(attnw, rows, cols, dtype):
     assert attnw.query_status() == 0
 
 
+@pytest.mark.parametrize("rows,cols", [(3, 8), (257, 100), (40, 260), (9, 1024), (5, 4096), (3, 8196), (2, 32768), (600, 512)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_recomputing_form_matches_oracle(attnw, rows, cols, dtype):
+    # the "recomputing" form of Section VI-A on row lengths the default serves from registers
+    S = inputs.normal_f32(11, rows * 137 + cols, rows * cols, 3.0).reshape(rows, cols)
+    raw, P, g = guarded_empty((rows, cols), dtype)
+    attnw.set_rows_variant("recomputing")
+    try:
+        attnw.softmax_rows(torch.from_numpy(S).cuda(), P=P)
+        torch.cuda.synchronize()
+    finally:
+        attnw.set_rows_variant("auto")
+    assert_guards_intact(raw, g)
+    assert_close_to_oracle(P, oracle.softmax_rows(S), f"recomputing rows={rows} cols={cols}")
+    assert attnw.query_status() == 0
+
+
+def test_caching_only_refuses_rows_beyond_the_register_tier(attnw):
+    S = torch.zeros((1, 40000), dtype=torch.float32, device="cuda")
+    attnw.set_rows_variant("caching")
+    try:
+        with pytest.raises(attnw.AttnwError) as e:
+            attnw.softmax_rows(S)
+        assert e.value.code == 4
+    finally:
+        attnw.set_rows_variant("auto")
+
+
 def test_in_place_f32(attnw):
     S = inputs.normal_f32(12, 1, 50 * 4096, 3.0).reshape(50, 4096)
     buf = torch.from_numpy(S).cuda()
