@@ -505,6 +505,8 @@ def run_ours(args):
             torch.cuda.empty_cache()
         other["c4_recomputing"] = secondary_config(binding, inputs, "c4", peaks, rows_variant="recomputing")
         torch.cuda.empty_cache()
+        other["c4_recomputing_registers"] = secondary_config(binding, inputs, "c4", peaks, rows_variant="recomputing_registers")
+        torch.cuda.empty_cache()
         other["attention_c3"] = attention_config(binding, inputs, "c3", peaks)
         torch.cuda.empty_cache()
         other["project_qk_c3"] = projection_config(binding, inputs, "c3", peaks)

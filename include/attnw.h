@@ -140,8 +140,11 @@ int softmax_rows_f32(const void* S, void* P, long long rows, long long cols, voi
  *   0  by row length (default): rows of up to 32768 columns are read once and kept in registers ("caching", one
  *      exponential per element); longer rows are read twice and their exponentials recomputed
  *   1  caching only: a call with cols > 32768 returns ATTNW_ERR_UNSUPPORTED
- *   2  recomputing for every row length: first read for the running maximum and sum, second read (mostly from L2)
- *      recomputes the exponentials - two exponentials and two reads per element, nothing kept on chip
+ *   2  recomputing for every row length, nothing kept on chip: rows of up to 32768 columns are read three times
+ *      (maximum; sum of exponentials; exponentials again for the output - the second and third read come from
+ *      L1 / L2), longer rows twice as under 0
+ *   3  recomputing from registers: rows of up to 32768 columns are read once, the SCORES are kept in registers and
+ *      every exponential is computed twice (for the sum, then for the output); longer rows: ATTNW_ERR_UNSUPPORTED
  * Returns ATTNW_ERR_BAD_SHAPE for any other value.
  */
 int attnw_set_rows_variant(int variant);

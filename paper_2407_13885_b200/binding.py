@@ -81,11 +81,12 @@ def set_fused_variant(variant: str | int) -> None:
     _check(lib.attnw_set_fused_variant(code), "attnw_set_fused_variant")
 
 
-ROWS_VARIANTS = {"auto": 0, "caching": 1, "recomputing": 2}
+ROWS_VARIANTS = {"auto": 0, "caching": 1, "recomputing": 2, "recomputing_registers": 3}
 
 
 def set_rows_variant(variant: str | int) -> None:
-    """Selects the form of ``softmax_rows``: "auto" (by row length), "caching" or "recomputing" (Section VI-A)."""
+    """Selects the form of ``softmax_rows``: "auto" (by row length), "caching", "recomputing" (second read) or
+    "recomputing_registers" (Section VI-A)."""
     code = ROWS_VARIANTS[variant] if isinstance(variant, str) else int(variant)
     _check(lib.attnw_set_rows_variant(code), "attnw_set_rows_variant")
 

@@ -27,7 +27,7 @@ constexpr int kMaxDevices = 64;
 constexpr int kVersion = 100;  // 0.1.0
 
 std::atomic<long long> g_launches{0};
-std::atomic<int> g_rows_variant{0};   // 0 = tier by row length, 1 = caching (register tier only), 2 = recomputing
+std::atomic<int> g_rows_variant{0};   // 0 = tier by row length, 1 = caching (register tier only), 2 = recomputing with a second read, 3 = recomputing from registers
 std::atomic<int> g_attn_variant{0};   // 0 = default (one pass), 1 = two-pass, 2 = one pass
 std::atomic<int> g_fused_variant{0};  // 0 = choose by shape, 1 = two-pass, 2 = SRAM-resident, 3 = SRAM-resident, owner-reduce exchange
 constexpr double kTwoPassPerSm = 0.9;  // measured: per-SM throughput of the two-pass kernel relative to the resident one
@@ -525,9 +525,9 @@ int rows_entry(const void* S, void* P, long long rows, long long cols, void* str
     rc = current_device(&dev);
     if (rc != ATTNW_OK) return rc;
     const int variant = g_rows_variant.load(std::memory_order_relaxed);
-    if (variant == 1 && cols > kSoftmaxRowsRegTierMaxCols) return ATTNW_ERR_UNSUPPORTED;
+    if ((variant == 1 || variant == 3) && cols > kSoftmaxRowsRegTierMaxCols) return ATTNW_ERR_UNSUPPORTED;
     cudaError_t e = softmax_rows_launch<OutT>(static_cast<const float*>(S), static_cast<OutT*>(P), rows, cols,
-                                              dev->sm_count, static_cast<cudaStream_t>(stream), variant == 2);
+                                              dev->sm_count, static_cast<cudaStream_t>(stream), variant == 3 ? 1 : (variant == 2 ? 2 : 0));
     if (e != cudaSuccess) return ATTNW_ERR_CUDA;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return ATTNW_OK;
@@ -607,7 +607,7 @@ int attnw_project_qk(const void* X, const void* Wq, const void* Wk, void* Q, voi
 }
 
 int attnw_set_rows_variant(int variant) {
-    if (variant < 0 || variant > 2) return ATTNW_ERR_BAD_SHAPE;
+    if (variant < 0 || variant > 3) return ATTNW_ERR_BAD_SHAPE;
     g_rows_variant.store(variant, std::memory_order_relaxed);
     return ATTNW_OK;
 }

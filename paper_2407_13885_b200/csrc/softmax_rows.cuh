@@ -22,6 +22,13 @@ __device__ __forceinline__ float sr_ex2(float x) {
     return y;
 }
 
+// A 16-byte load the compiler must issue each time it is written (the re-reading form reads a row three times).
+__device__ __forceinline__ float4 sr_reload4(const float4* p) {
+    float4 v;
+    asm volatile("ld.global.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
+    return v;
+}
+
 template <typename OutT>
 __device__ __forceinline__ void sr_store4(OutT* dst, float a, float b, float c, float d);
 
@@ -67,7 +74,11 @@ __device__ __forceinline__ float sr_row_reduce(float v, float* red) {
 //
 // Register tier: TPR threads per row, VPT float4 vectors per thread, row kept in registers.
 // A CTA has max(TPR, 256) threads and handles CTA_THREADS / TPR rows per sweep.
-template <int TPR, int VPT, typename OutT>
+// MODE 0: the registers keep the exponentials ("caching", Section VI-A).  MODE 1: they keep the scores and every
+// exponential is computed twice, once for the sum and once for the output ("recomputing" without its extra reads).
+// MODE 2: nothing is kept: the row is read for the maximum, read again for the sum and read a third time for the
+// output ("recomputing" as Section VI-A states it; the second and third read come from L1 / L2).
+template <int TPR, int VPT, typename OutT, int MODE = 0>
 __global__ void __launch_bounds__((TPR > 256 ? TPR : 256))
 softmax_rows_reg_kernel(const float* S, OutT* P, long long rows, int cols) {
     constexpr int kThreads = TPR > 256 ? TPR : 256;
@@ -90,7 +101,7 @@ softmax_rows_reg_kernel(const float* S, OutT* P, long long rows, int cols) {
         for (int k = 0; k < VPT; ++k) {
             const int idx = sub + k * TPR;
             if (row_ok && idx < nvec) {
-                v[k] = __ldcs(src + idx);
+                v[k] = MODE == 2 ? sr_reload4(src + idx) : __ldcs(src + idx);
                 m = fmaxf(m, fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w)));
             } else {
                 v[k] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
@@ -102,11 +113,14 @@ softmax_rows_reg_kernel(const float* S, OutT* P, long long rows, int cols) {
         // (x - m) first: the difference is exact near the maximum, so a constant row gives exactly 1.
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
-            v[k].x = sr_ex2((v[k].x - m) * kLog2e);
-            v[k].y = sr_ex2((v[k].y - m) * kLog2e);
-            v[k].z = sr_ex2((v[k].z - m) * kLog2e);
-            v[k].w = sr_ex2((v[k].w - m) * kLog2e);
-            l += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+            if constexpr (MODE == 2) {  // second read
+                const int idx = sub + k * TPR;
+                if (row_ok && idx < nvec) v[k] = sr_reload4(src + idx);
+            }
+            const float4 e = make_float4(sr_ex2((v[k].x - m) * kLog2e), sr_ex2((v[k].y - m) * kLog2e),
+                                         sr_ex2((v[k].z - m) * kLog2e), sr_ex2((v[k].w - m) * kLog2e));
+            l += (e.x + e.y) + (e.z + e.w);
+            if constexpr (MODE == 0) v[k] = e;
         }
         l = sr_row_reduce<TPR, false>(l, red_sum);
         const float inv = 1.0f / l;
@@ -114,6 +128,18 @@ softmax_rows_reg_kernel(const float* S, OutT* P, long long rows, int cols) {
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             const int idx = sub + k * TPR;
+            if constexpr (MODE == 2) {  // third read
+                if (row_ok && idx < nvec) v[k] = sr_reload4(src + idx);
+            }
+            if constexpr (MODE != 0) {
+                // asm volatile keeps the compiler from reusing the first pass's exponentials
+                float4 e;
+                asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.x) : "f"((v[k].x - m) * kLog2e));
+                asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.y) : "f"((v[k].y - m) * kLog2e));
+                asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.z) : "f"((v[k].z - m) * kLog2e));
+                asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.w) : "f"((v[k].w - m) * kLog2e));
+                v[k] = e;
+            }
             if (row_ok && idx < nvec)
                 sr_store4<OutT>(dst + 4ll * idx, v[k].x * inv, v[k].y * inv, v[k].z * inv, v[k].w * inv);
         }
@@ -176,41 +202,47 @@ softmax_rows_stream_kernel(const float* S, OutT* P, long long rows, long long co
 // Host-side tier selection; returns the cudaError_t of the launch.
 template <int TPR, int VPT, typename OutT>
 inline cudaError_t sr_launch_reg(const float* S, OutT* P, long long rows, int cols, int sm_count,
-                                 cudaStream_t stream) {
+                                 cudaStream_t stream, int mode) {
     constexpr int kThreads = TPR > 256 ? TPR : 256;
     constexpr int kRowsPerCta = kThreads / TPR;
     const long long sweeps = (rows + kRowsPerCta - 1) / kRowsPerCta;
     const long long cap = static_cast<long long>(sm_count) * 64;  // enough CTAs to fill every SM several times
     const unsigned grid = static_cast<unsigned>(sweeps < cap ? sweeps : cap);
-    softmax_rows_reg_kernel<TPR, VPT, OutT><<<grid, kThreads, 0, stream>>>(S, P, rows, cols);
+    if (mode == 1)
+        softmax_rows_reg_kernel<TPR, VPT, OutT, 1><<<grid, kThreads, 0, stream>>>(S, P, rows, cols);
+    else if (mode == 2)
+        softmax_rows_reg_kernel<TPR, VPT, OutT, 2><<<grid, kThreads, 0, stream>>>(S, P, rows, cols);
+    else
+        softmax_rows_reg_kernel<TPR, VPT, OutT><<<grid, kThreads, 0, stream>>>(S, P, rows, cols);
     return cudaGetLastError();
 }
 
 constexpr long long kSoftmaxRowsRegTierMaxCols = 32768;
 
-// recomputing: take the streaming tier whatever the row length (the "recomputing" form of Section VI-A on request)
+// mode: 0 caching, 1 recomputing from registers, 2 recomputing with re-reads (see the register-tier kernel); rows
+// beyond the register tier always take the streaming kernel, which is a recomputing form with one extra read
 template <typename OutT>
 inline cudaError_t softmax_rows_launch(const float* S, OutT* P, long long rows, long long cols, int sm_count,
-                                       cudaStream_t stream, bool recomputing = false) {
+                                       cudaStream_t stream, int mode = 0) {
     const long long nvec = cols / 4;
-    if (recomputing || cols > kSoftmaxRowsRegTierMaxCols) {
+    if (cols > kSoftmaxRowsRegTierMaxCols) {
         const long long cap = static_cast<long long>(sm_count) * 4;
         const unsigned grid = static_cast<unsigned>(rows < cap ? rows : cap);
         softmax_rows_stream_kernel<OutT><<<grid, 1024, 0, stream>>>(S, P, rows, cols);
         return cudaGetLastError();
     }
     const int c = static_cast<int>(cols);
-    if (nvec <= 8) return sr_launch_reg<8, 1, OutT>(S, P, rows, c, sm_count, stream);
-    if (nvec <= 16) return sr_launch_reg<8, 2, OutT>(S, P, rows, c, sm_count, stream);
-    if (nvec <= 32) return sr_launch_reg<8, 4, OutT>(S, P, rows, c, sm_count, stream);
-    if (nvec <= 64) return sr_launch_reg<32, 2, OutT>(S, P, rows, c, sm_count, stream);
-    if (nvec <= 128) return sr_launch_reg<32, 4, OutT>(S, P, rows, c, sm_count, stream);
-    if (nvec <= 256) return sr_launch_reg<32, 8, OutT>(S, P, rows, c, sm_count, stream);
-    if (nvec <= 512) return sr_launch_reg<256, 2, OutT>(S, P, rows, c, sm_count, stream);
-    if (nvec <= 1024) return sr_launch_reg<256, 4, OutT>(S, P, rows, c, sm_count, stream);
-    if (nvec <= 2048) return sr_launch_reg<256, 8, OutT>(S, P, rows, c, sm_count, stream);
-    if (nvec <= 4096) return sr_launch_reg<1024, 4, OutT>(S, P, rows, c, sm_count, stream);
-    return sr_launch_reg<1024, 8, OutT>(S, P, rows, c, sm_count, stream);
+    if (nvec <= 8) return sr_launch_reg<8, 1, OutT>(S, P, rows, c, sm_count, stream, mode);
+    if (nvec <= 16) return sr_launch_reg<8, 2, OutT>(S, P, rows, c, sm_count, stream, mode);
+    if (nvec <= 32) return sr_launch_reg<8, 4, OutT>(S, P, rows, c, sm_count, stream, mode);
+    if (nvec <= 64) return sr_launch_reg<32, 2, OutT>(S, P, rows, c, sm_count, stream, mode);
+    if (nvec <= 128) return sr_launch_reg<32, 4, OutT>(S, P, rows, c, sm_count, stream, mode);
+    if (nvec <= 256) return sr_launch_reg<32, 8, OutT>(S, P, rows, c, sm_count, stream, mode);
+    if (nvec <= 512) return sr_launch_reg<256, 2, OutT>(S, P, rows, c, sm_count, stream, mode);
+    if (nvec <= 1024) return sr_launch_reg<256, 4, OutT>(S, P, rows, c, sm_count, stream, mode);
+    if (nvec <= 2048) return sr_launch_reg<256, 8, OutT>(S, P, rows, c, sm_count, stream, mode);
+    if (nvec <= 4096) return sr_launch_reg<1024, 4, OutT>(S, P, rows, c, sm_count, stream, mode);
+    return sr_launch_reg<1024, 8, OutT>(S, P, rows, c, sm_count, stream, mode);
 }
 
 }  // namespace attnw

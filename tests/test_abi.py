@@ -119,9 +119,9 @@ def test_fused_variant_knob(lib):
 
 
 def test_rows_variant_knob(lib):
-    assert lib.attnw_set_rows_variant(3) == 2
+    assert lib.attnw_set_rows_variant(4) == 2
     assert lib.attnw_set_rows_variant(-1) == 2
-    for v in (1, 2, 0):
+    for v in (1, 2, 3, 0):
         assert lib.attnw_set_rows_variant(v) == 0
 
 

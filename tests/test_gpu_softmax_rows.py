@@ -36,11 +36,12 @@ def test_rows_match_oracle(attnw, rows, cols, dtype):
 
 @pytest.mark.parametrize("rows,cols", [(3, 8), (257, 100), (40, 260), (9, 1024), (5, 4096), (3, 8196), (2, 32768), (600, 512)])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
-def test_recomputing_form_matches_oracle(attnw, rows, cols, dtype):
+@pytest.mark.parametrize("form", ["recomputing", "recomputing_registers"])
+def test_recomputing_form_matches_oracle(attnw, rows, cols, dtype, form):
     # the "recomputing" form of Section VI-A on row lengths the default serves from registers
     S = inputs.normal_f32(11, rows * 137 + cols, rows * cols, 3.0).reshape(rows, cols)
     raw, P, g = guarded_empty((rows, cols), dtype)
-    attnw.set_rows_variant("recomputing")
+    attnw.set_rows_variant(form)
     try:
         attnw.softmax_rows(torch.from_numpy(S).cuda(), P=P)
         torch.cuda.synchronize()
