@@ -137,9 +137,12 @@ int softmax_rows_f32(const void* S, void* P, long long rows, long long cols, voi
 
 /*
  * Which form of the row Softmax softmax_rows uses (process-wide; Section VI-A compares the two on its hardware):
- *   0  by row length (default): rows of up to 32768 columns are read once and kept in registers ("caching", one
+ *   0  by row length (default): rows of up to 32768 columns are read once and kept in registers, rows of up to
+ *      49152 columns are read once and kept in the shared memory of one or two CTAs (both "caching": one
  *      exponential per element); longer rows are read twice and their exponentials recomputed
- *   1  caching only: a call with cols > 32768 returns ATTNW_ERR_UNSUPPORTED
+ *   1  caching only: rows of up to 393216 columns are kept in the shared memory of a thread-block cluster of up to
+ *      16 CTAs that exchange local maxima and sums through distributed shared memory; a call with cols > 393216
+ *      returns ATTNW_ERR_UNSUPPORTED
  *   2  recomputing for every row length, nothing kept on chip: rows of up to 32768 columns are read three times
  *      (maximum; sum of exponentials; exponentials again for the output - the second and third read come from
  *      L1 / L2), longer rows twice as under 0

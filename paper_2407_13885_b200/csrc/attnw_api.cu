@@ -18,6 +18,7 @@
 #include "project_qk.cuh"
 #include "attnw_resident.cuh"
 #include "softmax_rows.cuh"
+#include "softmax_rows_smem.cuh"
 
 namespace {
 
@@ -525,7 +526,21 @@ int rows_entry(const void* S, void* P, long long rows, long long cols, void* str
     rc = current_device(&dev);
     if (rc != ATTNW_OK) return rc;
     const int variant = g_rows_variant.load(std::memory_order_relaxed);
-    if ((variant == 1 || variant == 3) && cols > kSoftmaxRowsRegTierMaxCols) return ATTNW_ERR_UNSUPPORTED;
+    if (variant == 3 && cols > kSoftmaxRowsRegTierMaxCols) return ATTNW_ERR_UNSUPPORTED;
+    if (variant == 1 && cols > srs::kMaxCols) return ATTNW_ERR_UNSUPPORTED;
+    // Rows beyond the register tier can be kept in the shared memory of a CTA or of a cluster (caching form).  By
+    // default that is done where it is the faster way: up to clusters of two (49152 columns); with larger clusters
+    // the two cluster barriers per row cost more than the second read of the two-read kernel saves.
+    const int smem_ctas = cols > kSoftmaxRowsRegTierMaxCols ? srs::cluster_ctas_for(cols) : 0;
+    if ((variant == 1 && smem_ctas > 0) || (variant == 0 && smem_ctas > 0 && smem_ctas <= 2)) {
+        if (srs::launch<OutT>(static_cast<const float*>(S), static_cast<OutT*>(P), rows, cols, dev->sm_count,
+                              static_cast<cudaStream_t>(stream)) == cudaSuccess) {
+            g_launches.fetch_add(1, std::memory_order_relaxed);
+            return ATTNW_OK;
+        }
+        (void)cudaGetLastError();  // no cluster of that size on this device: fall through to the two-read kernel
+        if (variant == 1) return ATTNW_ERR_UNSUPPORTED;
+    }
     cudaError_t e = softmax_rows_launch<OutT>(static_cast<const float*>(S), static_cast<OutT*>(P), rows, cols,
                                               dev->sm_count, static_cast<cudaStream_t>(stream), variant == 3 ? 1 : (variant == 2 ? 2 : 0));
     if (e != cudaSuccess) return ATTNW_ERR_CUDA;

@@ -209,6 +209,17 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
     return r;
 }
+// 4-byte store into a peer CTA's shared memory (made visible by the cluster barrier that follows).
+__device__ __forceinline__ void st_cluster_f32(uint32_t remote_addr, float value) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote_addr), "f"(value) : "memory");
+}
+// Untiled bulk copy global -> this CTA's shared memory; both addresses 16-byte aligned, bytes a multiple of 16;
+// the mbarrier receives `bytes` of complete_tx.
+__device__ __forceinline__ void bulk_load_1d(uint32_t smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_dst),
+                 "l"(gmem_src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
 // 8-byte store into a peer CTA's shared memory; the peer's mbarrier receives 8 bytes of complete_tx.
 __device__ __forceinline__ void st_async_b64(uint32_t remote_addr, uint64_t value, uint32_t remote_mbar) {
     asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b64 [%0], %1, [%2];" ::"r"(remote_addr),

@@ -1,0 +1,195 @@
+// Row Softmax for rows too long for the register tier (Section VI, Eq. 1; "caching" form of Section VI-A): the row is
+// read from HBM once and kept in SHARED memory - of one CTA, or, beyond a CTA's share, of a thread-block cluster whose
+// CTAs hold consecutive slices of the row and exchange their local maxima and sums through distributed shared memory,
+// as the cores of the paper's Softmax kernel do across the chip (Section VI-B).  One exponential per element.
+//
+// Per row and CTA: one bulk asynchronous copy brings the slice in (at most 96 KB, so two CTAs share an SM and one
+// row's copy and barriers overlap the other's arithmetic and stores; two buffers in one CTA of 1024 threads were
+// slower: the per-row barriers, not the copy, are what has to be hidden); pass 1 over shared memory: maximum;
+// exchange; pass 2: e = 2^((x - M) log2 e) written back to shared memory, sum; exchange; pass 3: e / L -> P
+// (coalesced streaming stores).
+#pragma once
+#include "attnw_fused.cuh"
+#include "softmax_rows.cuh"
+
+namespace attnw {
+namespace srs {
+
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / 32;
+constexpr int kSliceMaxCols = 24576;                 // 96 KB of float32 per CTA
+constexpr int kMaxCluster = 16;
+constexpr long long kMaxCols = static_cast<long long>(kSliceMaxCols) * kMaxCluster;  // 393216
+constexpr uint32_t kPieceBytes = 16384;              // one bulk copy instruction
+constexpr uint32_t kSiteRowLoad = 120;               // wait site (low byte of the status word)
+
+struct Control {
+    uint64_t full;                 // the slice of the current row has landed
+    float red[kWarps];             // block reduction
+    float xch[2][kMaxCluster];     // [0]: local maxima, [1]: local sums of every CTA of the cluster
+    uint32_t abort_flag;
+    uint32_t prior_failure;
+};
+constexpr int kControlBytes = 256;
+static_assert(sizeof(Control) <= kControlBytes, "control block must fit its slot");
+
+template <bool IS_MAX>
+__device__ __forceinline__ float block_reduce(float v, float* red) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float o = __shfl_xor_sync(0xffffffffu, v, off);
+        v = IS_MAX ? fmaxf(v, o) : v + o;
+    }
+    __syncthreads();  // red[] of the previous reduction has been read by everyone
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float acc = red[0];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) acc = IS_MAX ? fmaxf(acc, red[w]) : acc + red[w];
+    return acc;
+}
+
+// grid: n_clusters * C CTAs in clusters of C; cluster i takes rows i, i + n_clusters, ...; slice_cols columns per CTA
+// (a multiple of 4; the last CTA's slice may be shorter or empty).
+template <typename OutT>
+__global__ void __launch_bounds__(kThreads, 2)
+softmax_rows_smem_kernel(const float* S, OutT* P, long long rows, long long cols, int slice_cols, int C) {
+    extern __shared__ __align__(16) uint8_t srs_smem[];
+    Control* ctl = reinterpret_cast<Control*>(srs_smem);
+    float* x = reinterpret_cast<float*>(srs_smem + kControlBytes);
+    volatile uint32_t* abort_flag = &ctl->abort_flag;
+
+    const uint32_t rank = C > 1 ? ptx::cluster_ctarank() : 0u;
+    const long long n_clusters = gridDim.x / C;
+    const long long cluster = blockIdx.x / C;
+    const long long c0 = static_cast<long long>(rank) * slice_cols;  // first column of this CTA's slice
+    const int n = static_cast<int>(c0 >= cols ? 0 : (cols - c0 < slice_cols ? cols - c0 : slice_cols));  // its length
+    const int nvec = n >> 2;
+
+    if (threadIdx.x == 0) {
+        ctl->prior_failure = *reinterpret_cast<volatile unsigned int*>(&g_attnw_status);
+        ptx::mbar_init(&ctl->full, 1);
+        ctl->abort_flag = 0;
+        ptx::mbar_fence_init();
+    }
+    __syncthreads();
+    // A CTA that sees an earlier failure still takes part in every cluster barrier below, without touching memory.
+    bool ok = ctl->prior_failure == 0u;
+    if (C > 1) {  // peers' control blocks are initialised before anyone writes into them
+        ptx::cluster_arrive_release();
+        ptx::cluster_wait_acquire();
+    }
+
+    uint32_t it = 0;
+    for (long long row = cluster; row < rows; row += n_clusters, ++it) {
+        const float* src = S + row * cols + c0;
+        if (ok && threadIdx.x == 0 && n > 0) {
+            const uint32_t bytes = static_cast<uint32_t>(n) * 4u;
+            ptx::mbar_expect_tx(&ctl->full, bytes);
+            for (uint32_t off = 0; off < bytes; off += kPieceBytes)
+                ptx::bulk_load_1d(ptx::smem_u32(x) + off, reinterpret_cast<const uint8_t*>(src) + off,
+                                  bytes - off < kPieceBytes ? bytes - off : kPieceBytes, &ctl->full);
+        }
+        if (ok && n > 0) ok = fused_wait(&ctl->full, it & 1u, abort_flag, kSiteRowLoad);
+        ok = __syncthreads_and(ok);  // all or none of the CTA goes on
+
+        // ---- pass 1: maximum ----
+        float m = -INFINITY;
+        if (ok)
+            for (int i = threadIdx.x; i < nvec; i += kThreads) {
+                const float4 v = reinterpret_cast<const float4*>(x)[i];
+                m = fmaxf(m, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
+            }
+        m = block_reduce<true>(m, ctl->red);
+        if (C > 1) {
+            if (threadIdx.x < static_cast<unsigned>(C))
+                ptx::st_cluster_f32(ptx::map_to_cta(ptx::smem_u32(&ctl->xch[0][rank]), threadIdx.x), m);
+            ptx::cluster_arrive_release();
+            ptx::cluster_wait_acquire();
+            m = ctl->xch[0][0];
+            for (int c = 1; c < C; ++c) m = fmaxf(m, ctl->xch[0][c]);
+        }
+        if (!(m > -INFINITY)) m = 0.0f;  // nothing was read (a failure upstream): keeps inf - inf out
+
+        // ---- pass 2: exponentials (kept in shared memory), sum ----
+        float l = 0.0f;
+        if (ok)
+            for (int i = threadIdx.x; i < nvec; i += kThreads) {
+                float4 v = reinterpret_cast<float4*>(x)[i];
+                // (x - M) first: the difference is exact near the maximum, so a constant row gives exactly 1
+                v.x = sr_ex2((v.x - m) * kLog2e);
+                v.y = sr_ex2((v.y - m) * kLog2e);
+                v.z = sr_ex2((v.z - m) * kLog2e);
+                v.w = sr_ex2((v.w - m) * kLog2e);
+                reinterpret_cast<float4*>(x)[i] = v;
+                l += (v.x + v.y) + (v.z + v.w);
+            }
+        l = block_reduce<false>(l, ctl->red);
+        if (C > 1) {
+            if (threadIdx.x < static_cast<unsigned>(C))
+                ptx::st_cluster_f32(ptx::map_to_cta(ptx::smem_u32(&ctl->xch[1][rank]), threadIdx.x), l);
+            ptx::cluster_arrive_release();
+            ptx::cluster_wait_acquire();
+            l = ctl->xch[1][0];
+            for (int c = 1; c < C; ++c) l += ctl->xch[1][c];  // the same order in every CTA
+        }
+
+        // ---- pass 3: normalise and store (each thread re-reads exactly what it wrote in pass 2) ----
+        if (ok) {
+            const float inv = 1.0f / l;
+            OutT* dst = P + row * cols + c0;
+            for (int i = threadIdx.x; i < nvec; i += kThreads) {
+                const float4 v = reinterpret_cast<const float4*>(x)[i];
+                sr_store4<OutT>(dst + 4ll * i, v.x * inv, v.y * inv, v.z * inv, v.w * inv);
+            }
+        }
+        ptx::fence_proxy_async_smem();  // orders this row's accesses to the slice before the next bulk copy into it
+        __syncthreads();                // the slice is free for the next row's copy
+    }
+    if (C > 1) {  // no CTA leaves while a peer may still write into its control block
+        ptx::cluster_arrive_release();
+        ptx::cluster_wait_acquire();
+    }
+}
+
+// Clusters of how many CTAs a row of `cols` columns needs (a power of two), or 0 if it does not fit this tier.
+inline int cluster_ctas_for(long long cols) {
+    if (cols > kMaxCols) return 0;
+    int c = 1;
+    while (static_cast<long long>(c) * kSliceMaxCols < cols) c *= 2;
+    return c;
+}
+
+template <typename OutT>
+inline cudaError_t launch(const float* S, OutT* P, long long rows, long long cols, int sm_count, cudaStream_t stream) {
+    const int C = cluster_ctas_for(cols);
+    if (C == 0) return cudaErrorInvalidValue;
+    const int slice_cols = static_cast<int>(((cols / 4 + C - 1) / C) * 4);
+    const size_t smem = kControlBytes + static_cast<size_t>(slice_cols) * 4;
+    auto kernel = softmax_rows_smem_kernel<OutT>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    if (C > 8) {
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e != cudaSuccess) return e;
+    }
+    long long n_clusters = (2ll * sm_count) / C;  // two CTAs per SM
+    if (n_clusters < 1) n_clusters = 1;
+    if (n_clusters > rows) n_clusters = rows;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(n_clusters * C));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(C);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, S, P, rows, cols, slice_cols, C);
+}
+
+}  // namespace srs
+}  // namespace attnw

@@ -19,7 +19,10 @@ def attnw():
 # every kernel tier and both sides of each tier boundary, with ragged tails
 SHAPES = [(1, 4), (3, 8), (33, 36), (257, 100), (64, 128), (5, 132), (40, 260), (17, 1000), (9, 1024),
           (7, 1028), (6, 2052), (5, 4096), (4, 4100), (3, 8192), (3, 8196), (2, 16384), (2, 16388),
-          (2, 32768), (3, 32772), (2, 70000), (600, 512)]
+          (2, 32768), (3, 32772), (2, 70000), (600, 512),
+          # the shared-memory tier: one CTA, clusters of 2, 4, 8 and 16, more rows than clusters, its last column count;
+          # then the two-read tier beyond it
+          (5, 40000), (3, 49152), (2, 100000), (1, 196608), (300, 33000), (1, 393216), (2, 393220), (40, 98308)]
 
 
 @pytest.mark.parametrize("rows,cols", SHAPES)
@@ -52,13 +55,33 @@ def test_recomputing_form_matches_oracle(attnw, rows, cols, dtype, form):
     assert attnw.query_status() == 0
 
 
-def test_caching_only_refuses_rows_beyond_the_register_tier(attnw):
-    S = torch.zeros((1, 40000), dtype=torch.float32, device="cuda")
+@pytest.mark.parametrize("rows,cols", [(2, 70000), (2, 100000), (1, 196608), (40, 98308), (1, 393216)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_cluster_cached_rows_match_oracle(attnw, rows, cols, dtype):
+    # the caching form on request: the row lives in the shared memory of a cluster of 4, 8 or 16 CTAs
+    S = inputs.normal_f32(11, rows * 139 + cols, rows * cols, 3.0).reshape(rows, cols)
+    raw, P, g = guarded_empty((rows, cols), dtype)
+    attnw.set_rows_variant("caching")
+    try:
+        attnw.softmax_rows(torch.from_numpy(S).cuda(), P=P)
+        torch.cuda.synchronize()
+    finally:
+        attnw.set_rows_variant("auto")
+    assert_guards_intact(raw, g)
+    assert_close_to_oracle(P, oracle.softmax_rows(S), f"cluster-cached rows={rows} cols={cols}")
+    assert attnw.query_status() == 0
+
+
+def test_caching_only_refuses_rows_beyond_the_on_chip_tiers(attnw):
+    S = torch.zeros((1, 393220), dtype=torch.float32, device="cuda")
     attnw.set_rows_variant("caching")
     try:
         with pytest.raises(attnw.AttnwError) as e:
             attnw.softmax_rows(S)
         assert e.value.code == 4
+        P = attnw.softmax_rows(S[:, :40000].contiguous())   # kept in shared memory: still the caching form
+        torch.cuda.synchronize()
+        assert bool((P.float() == 1.0 / 40000).all()) or float((P.float() - 1.0 / 40000).abs().max()) < 1e-7
     finally:
         attnw.set_rows_variant("auto")
 
