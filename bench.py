@@ -218,9 +218,9 @@ def time_launches(fn, steps, warmup, stream_sync):
     return start.elapsed_time(stop)
 
 
-def secondary_config(binding, inputs, name, peaks, steps=20, warmup=3, rows_variant="auto"):
-    """Short kernel-only measurement of one of the other configurations (reported, not the headline).
-    ``rows_variant``: the form of softmax_rows (Section VI-A's caching / recomputing comparison)."""
+def secondary_config(binding, inputs, name, peaks, steps=20, warmup=3):
+    """Short kernel-only measurement of one of the other configurations (reported, not the headline).  For the row
+    Softmax the two recomputing forms of Section VI-A are timed on the same buffers as well (``forms_ms``)."""
     import torch
     w = inputs.WORKLOADS[name]
     if w.kind == "rows":
@@ -237,17 +237,25 @@ def secondary_config(binding, inputs, name, peaks, steps=20, warmup=3, rows_vari
         P = torch.empty((w.B, w.H, w.N, w.N), dtype=torch.bfloat16 if w.p_dtype == "bf16" else torch.float32,
                         device="cuda")
         fn = lambda: binding.attnw_fused(Q, K, w.scale, P=P)  # noqa: E731
-    binding.set_rows_variant(rows_variant)
-    try:
-        ms = time_launches(fn, steps, warmup, torch.cuda.synchronize) / steps
-    finally:
-        binding.set_rows_variant("auto")
+    ms = time_launches(fn, steps, warmup, torch.cuda.synchronize) / steps
+    forms = None
+    if w.kind == "rows":
+        forms = {"caching": ms}
+        for form in ("recomputing_registers", "recomputing"):
+            binding.set_rows_variant(form)
+            try:
+                forms[form] = time_launches(fn, steps, warmup, torch.cuda.synchronize) / steps
+            finally:
+                binding.set_rows_variant("auto")
     bytes_alg = w.in_bytes + w.p_bytes
     t_hbm = bytes_alg / (peaks["hbm_gbs"] * 1e9)
     t_flop = w.flops / (peaks["bf16_tflops"] * 1e12)
-    return {"elements_per_s": w.elements / (ms * 1e-3), "ms": ms, "achieved_gbs": bytes_alg / (ms * 1e-3) / 1e9,
-            "roofline_frac": max(t_hbm, t_flop) / (ms * 1e-3), "bound": "hbm" if t_hbm >= t_flop else "tensor",
-            "steps": steps}
+    out = {"elements_per_s": w.elements / (ms * 1e-3), "ms": ms, "achieved_gbs": bytes_alg / (ms * 1e-3) / 1e9,
+           "roofline_frac": max(t_hbm, t_flop) / (ms * 1e-3), "bound": "hbm" if t_hbm >= t_flop else "tensor",
+           "steps": steps}
+    if forms:
+        out["forms_ms"] = forms
+    return out
 
 
 def attention_config(binding, inputs, name, peaks, steps=20, warmup=3):
@@ -503,10 +511,6 @@ def run_ours(args):
         for name in ("c4", "c5", "c2"):
             other[name] = secondary_config(binding, inputs, name, peaks)
             torch.cuda.empty_cache()
-        other["c4_recomputing"] = secondary_config(binding, inputs, "c4", peaks, rows_variant="recomputing")
-        torch.cuda.empty_cache()
-        other["c4_recomputing_registers"] = secondary_config(binding, inputs, "c4", peaks, rows_variant="recomputing_registers")
-        torch.cuda.empty_cache()
         other["attention_c3"] = attention_config(binding, inputs, "c3", peaks)
         torch.cuda.empty_cache()
         other["project_qk_c3"] = projection_config(binding, inputs, "c3", peaks)
