@@ -123,3 +123,34 @@ def test_attention_argument_errors(attnw):
     with pytest.raises(attnw.AttnwError) as e:
         attnw.attn_fused(y, y, y, 0.1)
     assert e.value.code == 4
+
+
+def test_attention_full_size_sampled(attnw):
+    """The launch the benchmark times (B=4, H=32, N=4096, d=128, V drawn like the benchmark's): no element left
+    unwritten, every output inside the range of V, and oracle parity on sampled complete rows of every head."""
+    w = inputs.WORKLOADS["c3"]
+    q, k = inputs.make_qk(w)
+    q, k = q.reshape(w.B, w.H, w.N, w.d), k.reshape(w.B, w.H, w.N, w.d)
+    v = inputs.normal_bf16_bits(inputs.SEED, 2 * w.cfg_id + 100, w.B * w.H * w.N * w.d, 1.0).reshape(w.B, w.H, w.N, w.d)
+    O = torch.empty((w.B, w.H, w.N, w.d), dtype=torch.bfloat16, device="cuda")
+    O.view(torch.int16).fill_(-1)  # NaN pattern
+    V = bits_to_cuda_bf16(v)
+    attnw.attn_fused(bits_to_cuda_bf16(q), bits_to_cuda_bf16(k), V, w.scale, O=O)
+    torch.cuda.synchronize()
+    assert attnw.query_status() == 0
+    assert not bool(torch.isnan(O).any())
+    # a convex combination of the values of its head, up to the rounding the tolerance allows
+    v_hi = V.float().amax(dim=2, keepdim=True)
+    v_lo = V.float().amin(dim=2, keepdim=True)
+    slack = tolerance(v)
+    assert bool((O.float() <= v_hi + slack).all()) and bool((O.float() >= v_lo - slack).all())
+    rng = np.random.default_rng(3)
+    ids = []
+    for bh in range(w.B * w.H):
+        local = {0, 127, 128, w.N - 129, w.N - 1} | set(rng.integers(0, w.N, size=3).tolist())
+        ids += [bh * w.N + i for i in sorted(local)]
+    ids = np.array(ids, dtype=np.int64)
+    ref = oracle.attn(q, k, v, w.scale, row_ids=ids)
+    got = O.view(-1, w.d)[torch.from_numpy(ids).cuda()].float().cpu().numpy().astype(np.float64)
+    err = float(np.max(np.abs(got - ref)))
+    assert err <= tolerance(v), f"{err:.3e} > {tolerance(v):.3e}"

@@ -114,3 +114,41 @@ def test_projection_argument_errors(attnw):
     with pytest.raises(attnw.AttnwError) as e:
         attnw.project_qk(x, w, w, Q=q, K=q)
     assert e.value.code == 7
+
+
+def test_projection_full_size_sampled(attnw):
+    """The launch the benchmark times (B=4, N=4096, d_model=4096, H=32, d=128, inputs drawn like the benchmark's): no
+    element left unwritten and oracle parity on sampled complete rows of every head of Q and of K."""
+    w = inputs.WORKLOADS["c3"]
+    dm = w.H * w.d
+    x = inputs.normal_bf16_bits(inputs.SEED, 2 * w.cfg_id + 200, w.B * w.N * dm, 1.0).reshape(w.B, w.N, dm)
+    wq = inputs.normal_bf16_bits(inputs.SEED, 2 * w.cfg_id + 201, w.H * w.d * dm, dm ** -0.5).reshape(w.H, w.d, dm)
+    wk = inputs.normal_bf16_bits(inputs.SEED, 2 * w.cfg_id + 202, w.H * w.d * dm, dm ** -0.5).reshape(w.H, w.d, dm)
+    Q = torch.empty((w.B, w.H, w.N, w.d), dtype=torch.bfloat16, device="cuda")
+    K = torch.empty_like(Q)
+    Q.view(torch.int16).fill_(-1)  # NaN pattern
+    K.view(torch.int16).fill_(-1)
+    attnw.project_qk(bits_to_cuda_bf16(x), bits_to_cuda_bf16(wq), bits_to_cuda_bf16(wk), Q=Q, K=K)
+    torch.cuda.synchronize()
+    assert attnw.query_status() == 0
+    assert not bool(torch.isnan(Q).any()) and not bool(torch.isnan(K).any())
+    rng = np.random.default_rng(4)
+    ids = []
+    for bh in range(w.B * w.H):
+        local = {0, 255, 256, w.N - 1} | set(rng.integers(0, w.N, size=2).tolist())
+        ids += [bh * w.N + i for i in sorted(local)]
+    ids = np.array(ids, dtype=np.int64)
+    sel = torch.from_numpy(ids).cuda()
+    # the bound of check(), with the largest sum |x||w| of the sampled rows
+    ax = np.abs(inputs.bf16_bits_to_f32(x).astype(np.float64))
+    for got_t, wb in ((Q, wq), (K, wk)):
+        ref = oracle.project(x, wb, row_ids=ids)
+        got = got_t.view(-1, w.d)[sel].float().cpu().numpy().astype(np.float64)
+        aw = np.abs(inputs.bf16_bits_to_f32(wb).astype(np.float64))
+        mass = 0.0
+        for g in ids[::37]:   # a subset is enough for the bound's scale; the maximum over it is then doubled
+            n, h, b = g % w.N, (g // w.N) % w.H, g // (w.N * w.H)
+            mass = max(mass, float((aw[h] @ ax[b, n]).max()))
+        tol = 2.0 ** -8 * np.abs(ref) + (dm / 16 + 17) * 2.0 ** -24 * (2.0 * mass)
+        err = np.abs(got - ref)
+        assert np.all(err <= tol), (float(err.max()), float((err / tol).max()))
