@@ -528,11 +528,13 @@ int rows_entry(const void* S, void* P, long long rows, long long cols, void* str
     const int variant = g_rows_variant.load(std::memory_order_relaxed);
     if (variant == 3 && cols > kSoftmaxRowsRegTierMaxCols) return ATTNW_ERR_UNSUPPORTED;
     if (variant == 1 && cols > srs::kMaxCols) return ATTNW_ERR_UNSUPPORTED;
-    // Rows beyond the register tier can be kept in the shared memory of a CTA or of a cluster (caching form).  By
-    // default that is done where it is the faster way: up to clusters of two (49152 columns); with larger clusters
-    // the two cluster barriers per row cost more than the second read of the two-read kernel saves.
-    const int smem_ctas = cols > kSoftmaxRowsRegTierMaxCols ? srs::cluster_ctas_for(cols) : 0;
-    if ((variant == 1 && smem_ctas > 0) || (variant == 0 && smem_ctas > 0 && smem_ctas <= 2)) {
+    // Longer rows can be kept in the shared memory of a CTA or of a cluster (caching form).  By default that is done
+    // where it is the faster way (measured): with one CTA from 8192 columns on - there the register tier needs a whole
+    // CTA of 1024 threads per row and stops overlapping rows - and with a cluster of two beyond the register tier;
+    // with larger clusters the two cluster barriers per row cost more than the second read of the two-read kernel.
+    const int smem_ctas = cols > kSoftmaxRowsSmemTierMinCols ? srs::cluster_ctas_for(cols) : 0;
+    const bool smem_default = smem_ctas == 1 || (smem_ctas == 2 && cols > kSoftmaxRowsRegTierMaxCols);
+    if ((variant <= 1 && smem_default) || (variant == 1 && smem_ctas > 2)) {
         if (srs::launch<OutT>(static_cast<const float*>(S), static_cast<OutT*>(P), rows, cols, dev->sm_count,
                               static_cast<cudaStream_t>(stream)) == cudaSuccess) {
             g_launches.fetch_add(1, std::memory_order_relaxed);

@@ -13,10 +13,13 @@
 #include "softmax_rows.cuh"
 
 namespace attnw {
+
+constexpr long long kSoftmaxRowsSmemTierMinCols = 8192;  // rows longer than this may leave the register tier
+
 namespace srs {
 
-constexpr int kThreads = 512;
-constexpr int kWarps = kThreads / 32;
+constexpr int kMaxThreads = 512;  // CTAs of 512 threads (two per SM) or, for slices of up to 48 KB, 256 (four per SM)
+constexpr int kWarps = kMaxThreads / 32;
 constexpr int kSliceMaxCols = 24576;                 // 96 KB of float32 per CTA
 constexpr int kMaxCluster = 16;
 constexpr long long kMaxCols = static_cast<long long>(kSliceMaxCols) * kMaxCluster;  // 393216
@@ -33,7 +36,7 @@ struct Control {
 constexpr int kControlBytes = 256;
 static_assert(sizeof(Control) <= kControlBytes, "control block must fit its slot");
 
-template <bool IS_MAX>
+template <bool IS_MAX, int NT>
 __device__ __forceinline__ float block_reduce(float v, float* red) {
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
@@ -45,14 +48,14 @@ __device__ __forceinline__ float block_reduce(float v, float* red) {
     __syncthreads();
     float acc = red[0];
 #pragma unroll
-    for (int w = 1; w < kWarps; ++w) acc = IS_MAX ? fmaxf(acc, red[w]) : acc + red[w];
+    for (int w = 1; w < NT / 32; ++w) acc = IS_MAX ? fmaxf(acc, red[w]) : acc + red[w];
     return acc;
 }
 
 // grid: n_clusters * C CTAs in clusters of C; cluster i takes rows i, i + n_clusters, ...; slice_cols columns per CTA
 // (a multiple of 4; the last CTA's slice may be shorter or empty).
-template <typename OutT>
-__global__ void __launch_bounds__(kThreads, 2)
+template <typename OutT, int NT>
+__global__ void __launch_bounds__(NT, NT == 256 ? 4 : 2)
 softmax_rows_smem_kernel(const float* S, OutT* P, long long rows, long long cols, int slice_cols, int C) {
     extern __shared__ __align__(16) uint8_t srs_smem[];
     Control* ctl = reinterpret_cast<Control*>(srs_smem);
@@ -96,11 +99,11 @@ softmax_rows_smem_kernel(const float* S, OutT* P, long long rows, long long cols
         // ---- pass 1: maximum ----
         float m = -INFINITY;
         if (ok)
-            for (int i = threadIdx.x; i < nvec; i += kThreads) {
+            for (int i = threadIdx.x; i < nvec; i += NT) {
                 const float4 v = reinterpret_cast<const float4*>(x)[i];
                 m = fmaxf(m, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
             }
-        m = block_reduce<true>(m, ctl->red);
+        m = block_reduce<true, NT>(m, ctl->red);
         if (C > 1) {
             if (threadIdx.x < static_cast<unsigned>(C))
                 ptx::st_cluster_f32(ptx::map_to_cta(ptx::smem_u32(&ctl->xch[0][rank]), threadIdx.x), m);
@@ -114,7 +117,7 @@ softmax_rows_smem_kernel(const float* S, OutT* P, long long rows, long long cols
         // ---- pass 2: exponentials (kept in shared memory), sum ----
         float l = 0.0f;
         if (ok)
-            for (int i = threadIdx.x; i < nvec; i += kThreads) {
+            for (int i = threadIdx.x; i < nvec; i += NT) {
                 float4 v = reinterpret_cast<float4*>(x)[i];
                 // (x - M) first: the difference is exact near the maximum, so a constant row gives exactly 1
                 v.x = sr_ex2((v.x - m) * kLog2e);
@@ -124,7 +127,7 @@ softmax_rows_smem_kernel(const float* S, OutT* P, long long rows, long long cols
                 reinterpret_cast<float4*>(x)[i] = v;
                 l += (v.x + v.y) + (v.z + v.w);
             }
-        l = block_reduce<false>(l, ctl->red);
+        l = block_reduce<false, NT>(l, ctl->red);
         if (C > 1) {
             if (threadIdx.x < static_cast<unsigned>(C))
                 ptx::st_cluster_f32(ptx::map_to_cta(ptx::smem_u32(&ctl->xch[1][rank]), threadIdx.x), l);
@@ -138,7 +141,7 @@ softmax_rows_smem_kernel(const float* S, OutT* P, long long rows, long long cols
         if (ok) {
             const float inv = 1.0f / l;
             OutT* dst = P + row * cols + c0;
-            for (int i = threadIdx.x; i < nvec; i += kThreads) {
+            for (int i = threadIdx.x; i < nvec; i += NT) {
                 const float4 v = reinterpret_cast<const float4*>(x)[i];
                 sr_store4<OutT>(dst + 4ll * i, v.x * inv, v.y * inv, v.z * inv, v.w * inv);
             }
@@ -160,25 +163,23 @@ inline int cluster_ctas_for(long long cols) {
     return c;
 }
 
-template <typename OutT>
-inline cudaError_t launch(const float* S, OutT* P, long long rows, long long cols, int sm_count, cudaStream_t stream) {
-    const int C = cluster_ctas_for(cols);
-    if (C == 0) return cudaErrorInvalidValue;
-    const int slice_cols = static_cast<int>(((cols / 4 + C - 1) / C) * 4);
+template <typename OutT, int NT>
+inline cudaError_t launch_nt(const float* S, OutT* P, long long rows, long long cols, int sm_count, int C, int slice_cols,
+                             cudaStream_t stream) {
     const size_t smem = kControlBytes + static_cast<size_t>(slice_cols) * 4;
-    auto kernel = softmax_rows_smem_kernel<OutT>;
+    auto kernel = softmax_rows_smem_kernel<OutT, NT>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (e != cudaSuccess) return e;
     if (C > 8) {
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
     }
-    long long n_clusters = (2ll * sm_count) / C;  // two CTAs per SM
+    long long n_clusters = (static_cast<long long>(NT == 256 ? 4 : 2) * sm_count) / C;  // CTAs that fit at once
     if (n_clusters < 1) n_clusters = 1;
     if (n_clusters > rows) n_clusters = rows;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(n_clusters * C));
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(NT);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -189,6 +190,15 @@ inline cudaError_t launch(const float* S, OutT* P, long long rows, long long col
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, S, P, rows, cols, slice_cols, C);
+}
+
+template <typename OutT>
+inline cudaError_t launch(const float* S, OutT* P, long long rows, long long cols, int sm_count, cudaStream_t stream) {
+    const int C = cluster_ctas_for(cols);
+    if (C == 0) return cudaErrorInvalidValue;
+    const int slice_cols = static_cast<int>(((cols / 4 + C - 1) / C) * 4);
+    if (slice_cols <= 12288) return launch_nt<OutT, 256>(S, P, rows, cols, sm_count, C, slice_cols, stream);
+    return launch_nt<OutT, 512>(S, P, rows, cols, sm_count, C, slice_cols, stream);
 }
 
 }  // namespace srs
