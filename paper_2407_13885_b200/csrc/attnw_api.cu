@@ -529,11 +529,11 @@ int rows_entry(const void* S, void* P, long long rows, long long cols, void* str
     if (variant == 3 && cols > kSoftmaxRowsRegTierMaxCols) return ATTNW_ERR_UNSUPPORTED;
     if (variant == 1 && cols > srs::kMaxCols) return ATTNW_ERR_UNSUPPORTED;
     // Longer rows can be kept in the shared memory of a CTA or of a cluster (caching form).  By default that is done
-    // where it is the faster way (measured): with one CTA from 8192 columns on - there the register tier needs a whole
-    // CTA of 1024 threads per row and stops overlapping rows - and with a cluster of two beyond the register tier;
-    // with larger clusters the two cluster barriers per row cost more than the second read of the two-read kernel.
+    // where it is the faster way (measured): from 8192 columns on - there the register tier needs a whole CTA of 1024
+    // threads per row and stops overlapping rows - with one CTA or a cluster of two; with larger clusters the cluster
+    // barrier of every row costs more than the second read of the two-read kernel.
     const int smem_ctas = cols > kSoftmaxRowsSmemTierMinCols ? srs::cluster_ctas_for(cols) : 0;
-    const bool smem_default = smem_ctas == 1 || (smem_ctas == 2 && cols > kSoftmaxRowsRegTierMaxCols);
+    const bool smem_default = smem_ctas == 1 || smem_ctas == 2;
     if ((variant <= 1 && smem_default) || (variant == 1 && smem_ctas > 2)) {
         if (srs::launch<OutT>(static_cast<const float*>(S), static_cast<OutT*>(P), rows, cols, dev->sm_count,
                               static_cast<cudaStream_t>(stream)) == cudaSuccess) {

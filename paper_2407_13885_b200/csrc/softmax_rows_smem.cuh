@@ -5,8 +5,9 @@
 //
 // Per row and CTA: one bulk asynchronous copy brings the slice in (at most 96 KB, so two CTAs share an SM and one
 // row's copy and barriers overlap the other's arithmetic and stores; two buffers in one CTA of 1024 threads were
-// slower: the per-row barriers, not the copy, are what has to be hidden); pass 1 over shared memory: maximum;
-// exchange; pass 2: e = 2^((x - M) log2 e) written back to shared memory, sum; exchange; pass 3: e / L -> P
+// slower: the per-row barriers, not the copy, are what has to be hidden); pass 1 over shared memory: the slice's
+// maximum m_c; pass 2: e = 2^((x - m_c) log2 e) written back to shared memory, the slice's sum l_c; ONE exchange of
+// the pairs (m_c, l_c); M = max m_c, L = sum l_c 2^((m_c - M) log2 e); pass 3: e * 2^((m_c - M) log2 e) / L -> P
 // (coalesced streaming stores).
 #pragma once
 #include "attnw_fused.cuh"
@@ -29,11 +30,11 @@ constexpr uint32_t kSiteRowLoad = 120;               // wait site (low byte of t
 struct Control {
     uint64_t full;                 // the slice of the current row has landed
     float red[kWarps];             // block reduction
-    float xch[2][kMaxCluster];     // [0]: local maxima, [1]: local sums of every CTA of the cluster
+    float xch[2][2][kMaxCluster];  // [row parity][0: local maxima, 1: local sums] of every CTA of the cluster
     uint32_t abort_flag;
     uint32_t prior_failure;
 };
-constexpr int kControlBytes = 256;
+constexpr int kControlBytes = 512;
 static_assert(sizeof(Control) <= kControlBytes, "control block must fit its slot");
 
 template <bool IS_MAX, int NT>
@@ -96,7 +97,7 @@ softmax_rows_smem_kernel(const float* S, OutT* P, long long rows, long long cols
         if (ok && n > 0) ok = fused_wait(&ctl->full, it & 1u, abort_flag, kSiteRowLoad);
         ok = __syncthreads_and(ok);  // all or none of the CTA goes on
 
-        // ---- pass 1: maximum ----
+        // ---- pass 1: maximum of the slice ----
         float m = -INFINITY;
         if (ok)
             for (int i = threadIdx.x; i < nvec; i += NT) {
@@ -104,46 +105,50 @@ softmax_rows_smem_kernel(const float* S, OutT* P, long long rows, long long cols
                 m = fmaxf(m, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
             }
         m = block_reduce<true, NT>(m, ctl->red);
-        if (C > 1) {
-            if (threadIdx.x < static_cast<unsigned>(C))
-                ptx::st_cluster_f32(ptx::map_to_cta(ptx::smem_u32(&ctl->xch[0][rank]), threadIdx.x), m);
-            ptx::cluster_arrive_release();
-            ptx::cluster_wait_acquire();
-            m = ctl->xch[0][0];
-            for (int c = 1; c < C; ++c) m = fmaxf(m, ctl->xch[0][c]);
-        }
-        if (!(m > -INFINITY)) m = 0.0f;  // nothing was read (a failure upstream): keeps inf - inf out
+        const float mc = (m > -INFINITY) ? m : 0.0f;  // an empty slice (or a failure upstream): keeps inf - inf out
 
-        // ---- pass 2: exponentials (kept in shared memory), sum ----
+        // ---- pass 2: exponentials relative to the slice's maximum (kept in shared memory), their sum ----
         float l = 0.0f;
         if (ok)
             for (int i = threadIdx.x; i < nvec; i += NT) {
                 float4 v = reinterpret_cast<float4*>(x)[i];
-                // (x - M) first: the difference is exact near the maximum, so a constant row gives exactly 1
-                v.x = sr_ex2((v.x - m) * kLog2e);
-                v.y = sr_ex2((v.y - m) * kLog2e);
-                v.z = sr_ex2((v.z - m) * kLog2e);
-                v.w = sr_ex2((v.w - m) * kLog2e);
+                // (x - m) first: the difference is exact near the maximum, so a constant row gives exactly 1
+                v.x = sr_ex2((v.x - mc) * kLog2e);
+                v.y = sr_ex2((v.y - mc) * kLog2e);
+                v.z = sr_ex2((v.z - mc) * kLog2e);
+                v.w = sr_ex2((v.w - mc) * kLog2e);
                 reinterpret_cast<float4*>(x)[i] = v;
                 l += (v.x + v.y) + (v.z + v.w);
             }
         l = block_reduce<false, NT>(l, ctl->red);
+
+        // ---- one exchange of (maximum, sum) across the cluster; the row's maximum and sum; this slice's factor ----
+        float factor;
         if (C > 1) {
-            if (threadIdx.x < static_cast<unsigned>(C))
-                ptx::st_cluster_f32(ptx::map_to_cta(ptx::smem_u32(&ctl->xch[1][rank]), threadIdx.x), l);
+            const uint32_t par = it & 1u;  // two sets of slots: a fast CTA's next row does not overwrite what a slow one reads
+            if (threadIdx.x < static_cast<unsigned>(C)) {
+                ptx::st_cluster_f32(ptx::map_to_cta(ptx::smem_u32(&ctl->xch[par][0][rank]), threadIdx.x), m);
+                ptx::st_cluster_f32(ptx::map_to_cta(ptx::smem_u32(&ctl->xch[par][1][rank]), threadIdx.x), l);
+            }
             ptx::cluster_arrive_release();
             ptx::cluster_wait_acquire();
-            l = ctl->xch[1][0];
-            for (int c = 1; c < C; ++c) l += ctl->xch[1][c];  // the same order in every CTA
+            float M = ctl->xch[par][0][0];
+            for (int c = 1; c < C; ++c) M = fmaxf(M, ctl->xch[par][0][c]);
+            if (!(M > -INFINITY)) M = 0.0f;
+            float L = 0.0f;
+            for (int c = 0; c < C; ++c)  // the same order in every CTA; an empty slice has sum 0 and maximum -inf
+                L += ctl->xch[par][1][c] * sr_ex2((ctl->xch[par][0][c] - M) * kLog2e);
+            factor = sr_ex2((mc - M) * kLog2e) / L;
+        } else {
+            factor = 1.0f / l;
         }
 
-        // ---- pass 3: normalise and store (each thread re-reads exactly what it wrote in pass 2) ----
+        // ---- pass 3: scale and store (each thread re-reads exactly what it wrote in pass 2) ----
         if (ok) {
-            const float inv = 1.0f / l;
             OutT* dst = P + row * cols + c0;
             for (int i = threadIdx.x; i < nvec; i += NT) {
                 const float4 v = reinterpret_cast<const float4*>(x)[i];
-                sr_store4<OutT>(dst + 4ll * i, v.x * inv, v.y * inv, v.z * inv, v.w * inv);
+                sr_store4<OutT>(dst + 4ll * i, v.x * factor, v.y * factor, v.z * factor, v.w * factor);
             }
         }
         ptx::fence_proxy_async_smem();  // orders this row's accesses to the slice before the next bulk copy into it
