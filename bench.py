@@ -218,6 +218,21 @@ def time_launches(fn, steps, warmup, stream_sync):
     return start.elapsed_time(stop)
 
 
+def reference_streams(steps=10, warmup=3):
+    """A plain device copy and a write-only fill of 2 GiB, timed in this run on this GPU (library kernels, context for the
+    roofline denominator only: the measured copy bandwidth of MEASURED_PEAKS.json stays the peak the fraction uses)."""
+    import torch
+    n = 1 << 29  # elements of 4 bytes
+    src = torch.empty(n, dtype=torch.float32, device="cuda")
+    dst = torch.empty(n, dtype=torch.float32, device="cuda")
+    src.fill_(1.0)
+    ms_copy = time_launches(lambda: dst.copy_(src), steps, warmup, torch.cuda.synchronize) / steps
+    ms_fill = time_launches(lambda: dst.fill_(3.0), steps, warmup, torch.cuda.synchronize) / steps
+    del src, dst
+    return {"copy_gbs": 2 * 4 * n / (ms_copy * 1e-3) / 1e9, "write_only_gbs": 4 * n / (ms_fill * 1e-3) / 1e9,
+            "bytes": 4 * n, "note": "torch copy_ (read + write) and fill_ (write only) of 2 GiB of float32, after the timed region"}
+
+
 def secondary_config(binding, inputs, name, peaks, steps=20, warmup=3):
     """Short kernel-only measurement of one of the other configurations (reported, not the headline).  For the row
     Softmax the two recomputing forms of Section VI-A are timed on the same buffers as well (``forms_ms``)."""
@@ -506,6 +521,8 @@ def run_ours(args):
         line["cpu_baseline"] = info
     if not args.no_secondary and world == 1:
         del P, Q, K
+        torch.cuda.empty_cache()
+        line["reference_streams"] = reference_streams()
         torch.cuda.empty_cache()
         other = {}
         for name in ("c4", "c5", "c2"):
