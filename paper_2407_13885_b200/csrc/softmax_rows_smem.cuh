@@ -19,7 +19,7 @@ constexpr long long kSoftmaxRowsSmemTierMinCols = 8192;  // rows longer than thi
 
 namespace srs {
 
-constexpr int kMaxThreads = 512;  // CTAs of 512 threads (two per SM) or, for slices of up to 48 KB, 256 (four per SM)
+constexpr int kMaxThreads = 512;  // CTAs of 512 threads (two per SM) or, for slices of up to 64 KB, 256 (three or four per SM)
 constexpr int kWarps = kMaxThreads / 32;
 constexpr int kSliceMaxCols = 24576;                 // 96 KB of float32 per CTA
 constexpr int kMaxCluster = 16;
@@ -179,7 +179,8 @@ inline cudaError_t launch_nt(const float* S, OutT* P, long long rows, long long 
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
         if (e != cudaSuccess) return e;
     }
-    long long n_clusters = (static_cast<long long>(NT == 256 ? 4 : 2) * sm_count) / C;  // CTAs that fit at once
+    const long long per_sm = NT == 256 ? (smem * 4 <= 224 * 1024 ? 4 : 3) : 2;
+    long long n_clusters = (per_sm * sm_count) / C;  // CTAs that fit at once
     if (n_clusters < 1) n_clusters = 1;
     if (n_clusters > rows) n_clusters = rows;
     cudaLaunchConfig_t cfg = {};
@@ -202,7 +203,7 @@ inline cudaError_t launch(const float* S, OutT* P, long long rows, long long col
     const int C = cluster_ctas_for(cols);
     if (C == 0) return cudaErrorInvalidValue;
     const int slice_cols = static_cast<int>(((cols / 4 + C - 1) / C) * 4);
-    if (slice_cols <= 12288) return launch_nt<OutT, 256>(S, P, rows, cols, sm_count, C, slice_cols, stream);
+    if (slice_cols <= 16384) return launch_nt<OutT, 256>(S, P, rows, cols, sm_count, C, slice_cols, stream);
     return launch_nt<OutT, 512>(S, P, rows, cols, sm_count, C, slice_cols, stream);
 }
 
