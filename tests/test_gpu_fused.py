@@ -243,6 +243,30 @@ def test_full_size_configs_sampled(attnw, name, variant):
     assert err <= TOL[torch.bfloat16]["abs"], f"{name}: max abs err {err:.3e}"
 
 
+@pytest.mark.parametrize("name", ["c3", "c5"])
+def test_full_size_configs_every_element(attnw, name):
+    """Every element of the launch the benchmark times against the oracle (2.1e9 elements each; the oracle takes
+    some ten seconds per configuration on the host's cores, one head - or 2048 rows of a head - at a time)."""
+    w = inputs.WORKLOADS[name]
+    q, k = inputs.make_qk(w)
+    q = q.reshape(w.B, w.H, w.N, w.d)
+    k = k.reshape(w.B, w.H, w.N, w.d)
+    P = attnw.attnw_fused(bits_to_cuda_bf16(q), bits_to_cuda_bf16(k), w.scale)
+    torch.cuda.synchronize()
+    assert attnw.query_status() == 0
+    flat = P.view(w.B * w.H, w.N, w.N)
+    qf, kf = q.reshape(w.B * w.H, 1, w.N, w.d), k.reshape(w.B * w.H, 1, w.N, w.d)
+    step = 2048
+    worst = 0.0
+    for bh in range(w.B * w.H):
+        for r0 in range(0, w.N, step):
+            ids = np.arange(r0, min(r0 + step, w.N), dtype=np.int64)
+            ref = oracle.attnw_rows(qf[bh:bh + 1], kf[bh:bh + 1], w.scale, ids)
+            got = flat[bh, r0:r0 + step].float().cpu().numpy().astype(np.float64)
+            worst = max(worst, float(np.max(np.abs(got - ref))))
+    assert worst <= TOL[torch.bfloat16]["abs"], f"{name}: max abs err over all elements {worst:.3e}"
+
+
 def test_device_side_argument_errors(attnw):
     q = torch.zeros((1, 1, 128, 64), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(attnw.AttnwError) as e:
