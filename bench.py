@@ -363,6 +363,14 @@ def run_profile_case(args):
         K = torch.empty_like(Q)
         fn = lambda: binding.project_qk(X, Wq, Wk, Q=Q, K=K)  # noqa: E731
         desc = f"attnw_project_qk B=1 N={w.N} d_model={dm} H={w.H} d={w.d}"
+    elif args.profile == "rows_long":
+        # rows beyond the register tier: kept in the shared memory of a cluster of two CTAs (32768 columns)
+        rows, cols = 4096, 32768
+        w = inputs.Workload("rows-long", "rows", rows=rows, cols=cols, sigma=3.0, cfg_id=4)
+        S = torch.from_numpy(inputs.make_scores(w, 0, rows)).cuda()
+        P = torch.empty((rows, cols), dtype=torch.bfloat16, device="cuda")
+        fn = lambda: binding.softmax_rows(S, P=P)  # noqa: E731
+        desc = f"softmax_rows rows={rows} cols={cols} (S {w.in_bytes >> 20} MiB, P {w.p_bytes >> 20} MiB)"
     else:
         base = inputs.WORKLOADS["c4"]
         rows = 8192
@@ -553,7 +561,7 @@ def main():
     ap.add_argument("--sustained-seconds", type=float, default=2.0)
     ap.add_argument("--variant", choices=["auto", "two_pass", "resident"], default="auto",
                     help="kernel behind attnw_fused (see attnw_set_fused_variant)")
-    ap.add_argument("--profile", choices=["fused", "rows", "attention", "project"], default=None,
+    ap.add_argument("--profile", choices=["fused", "rows", "rows_long", "attention", "project"], default=None,
                     help="run a reduced case of one kernel for an ncu capture instead of the benchmark")
     args = ap.parse_args()
     if args.impl == "reference":
