@@ -559,7 +559,7 @@ def main():
     ap.add_argument("--no-secondary", action="store_true")
     ap.add_argument("--no-sustained", action="store_true")
     ap.add_argument("--sustained-seconds", type=float, default=2.0)
-    ap.add_argument("--variant", choices=["auto", "two_pass", "resident"], default="auto",
+    ap.add_argument("--variant", choices=["auto", "two_pass", "resident", "gridrow"], default="auto",
                     help="kernel behind attnw_fused (see attnw_set_fused_variant)")
     ap.add_argument("--profile", choices=["fused", "rows", "rows_long", "attention", "project"], default=None,
                     help="run a reduced case of one kernel for an ncu capture instead of the benchmark")

@@ -117,6 +117,13 @@ int attnw_set_attn_variant(int variant);
  *   3  the same kernel with the exchange the paper leaves as future work (Section IX): the rows are dealt out to
  *      the CTAs of the cluster, the owner of a row receives its local maxima and sums, reduces them once and
  *      sends the global values to every CTA (reduce and broadcast) instead of every CTA reducing redundantly
+ *   4  grid-row kernel: the SRAM-resident design on a cooperative grid of one CTA per SM.  Consecutive ceil(N/256)
+ *      CTAs form a group (the cores of one grid row in Section VII) that owns a 128-row block; every CTA keeps its
+ *      128 x 256 slab of scores in half of its tensor memory, so two row blocks are in flight per CTA, and the local
+ *      row maxima and sums cross the group through L2 as tagged 16-byte messages in a per-device exchange area that
+ *      the library allocates on first use (cudaMalloc; never inside a stream capture).  Serves bfloat16 P and
+ *      N <= 4096; any other call then returns ATTNW_ERR_UNSUPPORTED.  Two such launches must not run on one device
+ *      at the same time (they share the exchange area); launches on one stream, or ordered by events, are fine.
  * Returns ATTNW_ERR_BAD_SHAPE for any other value.
  */
 int attnw_set_fused_variant(int variant);

@@ -71,12 +71,12 @@ def version() -> int:
     return int(lib.attnw_version())
 
 
-FUSED_VARIANTS = {"auto": 0, "two_pass": 1, "resident": 2, "resident_owner": 3}
+FUSED_VARIANTS = {"auto": 0, "two_pass": 1, "resident": 2, "resident_owner": 3, "gridrow": 4}
 
 
 def set_fused_variant(variant: str | int) -> None:
-    """Selects the kernel behind ``attnw_fused``: "auto" (by shape), "two_pass", "resident" or "resident_owner"
-    (the resident kernel with the reduce-and-broadcast exchange)."""
+    """Selects the kernel behind ``attnw_fused``: "auto" (by shape), "two_pass", "resident", "resident_owner"
+    (the resident kernel with the reduce-and-broadcast exchange) or "gridrow" (groups of CTAs of a cooperative grid)."""
     code = FUSED_VARIANTS[variant] if isinstance(variant, str) else int(variant)
     _check(lib.attnw_set_fused_variant(code), "attnw_set_fused_variant")
 

@@ -17,6 +17,7 @@
 #include "attn_onepass.cuh"
 #include "project_qk.cuh"
 #include "attnw_resident.cuh"
+#include "attnw_gridrow.cuh"
 #include "softmax_rows.cuh"
 #include "softmax_rows_smem.cuh"
 
@@ -43,6 +44,12 @@ struct DeviceInfo {
     // fork/join objects for launches that split a call over two kernels (created on first use)
     cudaStream_t side_stream = nullptr;
     cudaEvent_t fork_event = nullptr, join_event = nullptr;
+    // grid-row kernel: co-resident CTAs per head dimension (0 = not asked yet), the exchange area in device memory
+    // (created on first use, zeroed once) and the next unused message tag
+    int gridrow_ctas[2] = {};
+    uint4* gridrow_xchg = nullptr;
+    int gridrow_xchg_ctas = 0;
+    uint32_t gridrow_tag = 0;
 };
 std::mutex g_split_mutex;
 DeviceInfo g_devices[kMaxDevices];
@@ -303,6 +310,88 @@ int launch_resident(DeviceInfo* dev, const void* Q, const void* K, void* P, int 
                  : launch_resident_impl<D, 16, false>(dev, Q, K, P, BH, N, scale, stream);
 }
 
+// Grid-row kernel: a cooperative grid of one CTA per SM; consecutive ceil(N / 256) CTAs form a group that owns a
+// 128-row block and walks a contiguous part of the list of row blocks.  Returns ATTNW_ERR_UNSUPPORTED when the
+// device cannot hold a whole group at once.
+template <int D>
+int launch_gridrow(DeviceInfo* dev, const void* Q, const void* K, void* P, int BH, int N, float scale, cudaStream_t stream) {
+    using L = gr::Smem<D>;
+    auto kernel = gr::attnw_gridrow_kernel<D>;
+    CUtensorMap tm_q, tm_k, tm_p;
+    int rc = encode_3d(&tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Q, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, K, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_p, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, P, N, N, BH, 64, kTile);
+    if (rc != ATTNW_OK) return rc;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    const int group_ctas = (N + gr::kSlabCols - 1) / gr::kSlabCols;
+    const int row_blocks = (N + kTile - 1) / kTile;
+    const long long total_items = static_cast<long long>(BH) * row_blocks;
+    if (total_items > INT_MAX) return ATTNW_ERR_BAD_SHAPE;
+    uint4* xchg = nullptr;
+    uint32_t tag_base = 0;
+    int n_groups = 0;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        int& max_ctas = dev->gridrow_ctas[D == 128 ? 1 : 0];
+        if (max_ctas == 0) {
+            int per_sm = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, gr::kThreads, L::kDynamicBytes) != cudaSuccess ||
+                per_sm < 1) {
+                (void)cudaGetLastError();
+                max_ctas = -1;
+            } else {
+                max_ctas = dev->sm_count;  // one CTA per SM: the kernel takes all of tensor memory
+            }
+        }
+        if (max_ctas < group_ctas) return ATTNW_ERR_UNSUPPORTED;
+        n_groups = max_ctas / group_ctas;
+        if (n_groups > total_items) n_groups = static_cast<int>(total_items);
+        if (dev->gridrow_xchg == nullptr || dev->gridrow_xchg_ctas < max_ctas) {
+            // first use on this device: the exchange area, zero so that no entry carries a valid tag
+            if (dev->gridrow_xchg) cudaFree(dev->gridrow_xchg);
+            dev->gridrow_xchg = nullptr;
+            const size_t bytes = static_cast<size_t>(max_ctas) * gr::kXchgDepth * kTile * sizeof(uint4);
+            void* p = nullptr;
+            if (cudaMalloc(&p, bytes) != cudaSuccess || cudaMemset(p, 0, bytes) != cudaSuccess ||
+                cudaDeviceSynchronize() != cudaSuccess) {
+                (void)cudaGetLastError();
+                if (p) cudaFree(p);
+                return ATTNW_ERR_CUDA;
+            }
+            dev->gridrow_xchg = static_cast<uint4*>(p);
+            dev->gridrow_xchg_ctas = max_ctas;
+            dev->gridrow_tag = 0;
+        }
+        xchg = dev->gridrow_xchg;
+        // tags tag_base + 1 ... tag_base + (longest list) belong to this launch; 0 is never a tag
+        const uint32_t longest = static_cast<uint32_t>((total_items + n_groups - 1) / n_groups);
+        if (dev->gridrow_tag > 0xffffffffu - longest - 1u) dev->gridrow_tag = 0;
+        tag_base = dev->gridrow_tag;
+        dev->gridrow_tag += longest;
+    }
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;  // every CTA of the grid is resident at once, or the launch fails
+    attr[0].val.cooperative = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(gr::kThreads, 1, 1);
+    cfg.gridDim = dim3(static_cast<unsigned>(n_groups * group_ctas), 1, 1);
+    cfg.dynamicSmemBytes = L::kDynamicBytes;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const float scale_log2e = static_cast<float>(static_cast<double>(scale) * 1.4426950408889634074);
+    if (cudaLaunchKernelEx(&cfg, kernel, tm_q, tm_k, tm_p, N, static_cast<int>(total_items), group_ctas, n_groups, scale_log2e,
+                           xchg, tag_base) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTNW_OK;
+}
+
 template <int D>
 int launch_attn(const void* Q, const void* K, const void* V, void* O, int BH, int N, float scale, cudaStream_t stream) {
     using L = FusedSmem<D>;
@@ -427,6 +516,14 @@ int fused_entry(const void* Q, const void* K, void* P, int B, int H, int N, int 
     const int variant = g_fused_variant.load(std::memory_order_relaxed);
     const bool resident_fits = sizeof(OutT) == 2 && N <= kResidentMaxN;
     if ((variant == 2 || variant == 3) && !resident_fits) return ATTNW_ERR_UNSUPPORTED;
+    if (variant == 4) {
+        if constexpr (sizeof(OutT) == 2) {
+            if (N > gr::kMaxN) return ATTNW_ERR_UNSUPPORTED;
+            return (d == 64) ? launch_gridrow<64>(dev, Q, K, P, B * H, N, scale, s)
+                             : launch_gridrow<128>(dev, Q, K, P, B * H, N, scale, s);
+        }
+        return ATTNW_ERR_UNSUPPORTED;
+    }
     if (variant == 3) {
         if constexpr (sizeof(OutT) == 2)
             return (d == 64) ? launch_resident<64>(dev, Q, K, P, B * H, N, scale, s, true)
@@ -763,7 +860,7 @@ int attnw_query_status(void* stream, unsigned int* device_status) {
 }
 
 int attnw_set_fused_variant(int variant) {
-    if (variant < 0 || variant > 3) return ATTNW_ERR_BAD_SHAPE;
+    if (variant < 0 || variant > 4) return ATTNW_ERR_BAD_SHAPE;
     g_fused_variant.store(variant, std::memory_order_relaxed);
     return ATTNW_OK;
 }
@@ -796,10 +893,14 @@ int attnw_debug_cta_clock(long long* out) {
 }
 #endif
 #ifdef ATTNW_TIMELINE
+int attnw_debug_gt(unsigned long long* out) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return ATTNW_ERR_CUDA;
+    return cudaMemcpyFromSymbol(out, attnw::gr::g_attnw_gt, sizeof(unsigned long long) * 160 * 3 * 160) == cudaSuccess ? ATTNW_OK : ATTNW_ERR_CUDA;
+}
 // Debug builds only (-DATTNW_TIMELINE=<cta index>): copies the cycle stamps of that CTA to the host.
 int attnw_debug_timeline(long long* out) {
     if (cudaDeviceSynchronize() != cudaSuccess) return ATTNW_ERR_CUDA;
-    return cudaMemcpyFromSymbol(out, attnw::g_attnw_timeline, sizeof(long long) * 16 * 160) == cudaSuccess ? ATTNW_OK
+    return cudaMemcpyFromSymbol(out, attnw::g_attnw_timeline, sizeof(long long) * 32 * 160) == cudaSuccess ? ATTNW_OK
                                                                                                           : ATTNW_ERR_CUDA;
 }
 #endif

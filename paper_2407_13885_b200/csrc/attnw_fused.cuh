@@ -42,7 +42,7 @@ __device__ unsigned int g_attnw_status = 0;
 __device__ long long g_attnw_cta_clock[4096][4];  // per CTA: cycles, nanoseconds, SM id, start ns
 #endif
 #ifdef ATTNW_TIMELINE
-__device__ long long g_attnw_timeline[16][160];
+__device__ long long g_attnw_timeline[32][160];
 #define ATTNW_STAMP(ev, it)                                                                       \
     do {                                                                                          \
         if (blockIdx.x == ATTNW_TIMELINE && (it) < 160) g_attnw_timeline[ev][it] = clock64();     \

@@ -112,9 +112,9 @@ def test_rows_argument_errors_are_host_side(lib):
 
 
 def test_fused_variant_knob(lib):
-    assert lib.attnw_set_fused_variant(4) == 2
+    assert lib.attnw_set_fused_variant(5) == 2
     assert lib.attnw_set_fused_variant(-1) == 2
-    for v in (1, 2, 3, 0):
+    for v in (1, 2, 3, 4, 0):
         assert lib.attnw_set_fused_variant(v) == 0
 
 

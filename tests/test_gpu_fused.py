@@ -63,6 +63,22 @@ def test_resident_variant_matches_oracle(attnw, B, H, N, d, variant):
     assert_close_to_oracle(P, oracle.attnw(q, k, scale), f"{variant} B{B} H{H} N{N} d{d}")
 
 
+# The grid-row kernel: groups of 1..16 CTAs, ragged slabs (one or two slots in use in the last CTA), ragged row blocks,
+# lists that cross head boundaries inside a group, more groups than row blocks.
+GRIDROW_SHAPES = [(1, 1, 128, 64), (1, 1, 256, 128), (1, 2, 512, 128), (1, 3, 384, 64), (2, 2, 2048, 64),
+                  (1, 2, 4096, 128), (1, 1, 200, 128), (1, 1, 1160, 64), (1, 2, 2568, 128), (1, 1, 8, 64),
+                  (1, 1, 3080, 64), (3, 5, 640, 128), (1, 7, 1024, 64), (1, 40, 264, 64), (1, 3, 3848, 128)]
+
+
+@pytest.mark.parametrize("B,H,N,d", GRIDROW_SHAPES)
+def test_gridrow_variant_matches_oracle(attnw, B, H, N, d):
+    q, k = small_fused_inputs(B, H, N, d, stream=N + d + 11)
+    scale = float(np.float32(1.0 / math.sqrt(d)))
+    for _ in range(2):  # twice: the second launch finds the exchange area as the first one left it
+        P = run_fused(attnw, q, k, scale, torch.bfloat16, variant="gridrow")
+        assert_close_to_oracle(P, oracle.attnw(q, k, scale), f"gridrow B{B} H{H} N{N} d{d}")
+
+
 def test_default_choice_splits_a_call_over_both_kernels(attnw):
     # B*H = 32, N = 2048: 33 clusters of 4 leave 16 SMs idle and walk 16 rounds of row blocks, so the default
     # choice gives two heads to the two-pass kernel on a side stream; the whole of P must be there afterwards
