@@ -34,19 +34,18 @@ namespace attnw {
 namespace gr {
 
 constexpr int kSlabCols = 256;                       // key columns per CTA and row block
-#ifndef ATTNW_GR_SLOT_COLS
-#define ATTNW_GR_SLOT_COLS 128
-#endif
-constexpr int kSub = ATTNW_GR_SLOT_COLS;             // columns per MMA slot (the unit tensor memory is handed over in)
-constexpr int kSubsPerBlock = kSlabCols / kSub;
+constexpr int kSub = 128;                            // columns per MMA landing slot
+constexpr int kSubsPerBlock = kSlabCols / kSub;      // 2 landing slots = tensor-memory columns [0, 256)
+constexpr int kPackedCol0 = kSlabCols;               // packed exponentials: columns [256, 512), 128 per stream
+constexpr int kPackedCols = kSlabCols / 2;           // two f16 per 32-bit column
 constexpr int kBoxCols = 64;                         // columns of one staged store box (128 bytes of bf16)
 constexpr int kChunksPerBlock = kSlabCols / kChunk;  // 32-column chunks, each with its own offset
 #ifndef ATTNW_GR_THREADS
-#define ATTNW_GR_THREADS 608
+#define ATTNW_GR_THREADS 640
 #endif
 constexpr int kThreads = ATTNW_GR_THREADS;           // 8 exponential + 8 normalise warps, producer, MMA issuer, store issuer
 constexpr int kNormWarp0 = 8;
-constexpr int kNormGroups = (kThreads >= 608) ? 2 : 1;  // normalise warpgroups: one per stream, or one for both
+constexpr int kNormGroups = 2;                         // normalise warpgroups: one per stream, or one for both
 constexpr int kProducerWarpG = kNormWarp0 + 4 * kNormGroups;
 constexpr int kMmaWarpG = kProducerWarpG + 1;
 constexpr int kStoreWarpG = kProducerWarpG + 2;
@@ -90,7 +89,8 @@ static_assert(Smem<128>::kDynamicBytes <= 227 * 1024 && Smem<64>::kDynamicBytes 
 struct Barriers {
     uint64_t k_full, k_empty;
     uint64_t q_full[2], q_empty[2];
-    uint64_t s_full[2][kSubsPerBlock], slot_free[2][kSubsPerBlock];
+    uint64_t s_full[kSubsPerBlock], l_free[kSubsPerBlock];  // landing slots: scores ready / scores taken to registers
+    uint64_t pk_free[2][kSlabCols / kBoxCols];              // [stream][box]: the packed exponentials have been read
     uint64_t posted[2];
     uint64_t out_free[6], out_filled[6];
     uint32_t tmem_base;
@@ -161,14 +161,15 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     if (threadIdx.x == 0) {
         ptx::mbar_init(&bars->k_full, 1);
         ptx::mbar_init(&bars->k_empty, 1);
+        for (int j = 0; j < kSubsPerBlock; ++j) {
+            ptx::mbar_init(&bars->s_full[j], 1);
+            ptx::mbar_init(&bars->l_free[j], 8);  // one arrival per exponential warp
+        }
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(&bars->q_full[s], 1);
             ptx::mbar_init(&bars->q_empty[s], 1);
-            for (int j = 0; j < kSubsPerBlock; ++j) {
-                ptx::mbar_init(&bars->s_full[s][j], 1);
-                ptx::mbar_init(&bars->slot_free[s][j], 4);  // one arrival per normalise warp of the stream
-            }
-            ptx::mbar_init(&bars->posted[s], 8);            // one arrival per exponential warp
+            for (int b = 0; b < kSlabCols / kBoxCols; ++b) ptx::mbar_init(&bars->pk_free[s][b], 4);  // the stream's normalise warps
+            ptx::mbar_init(&bars->posted[s], 8);  // one arrival per exponential warp
         }
         for (int b = 0; b < kBoxes; ++b) {
             ptx::mbar_init(&bars->out_free[b], 1);
@@ -267,12 +268,12 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             }
             const bool last_of_head = (i + 1 == n_items) || ((gi + 1) / T != bh);
             for (int j = 0; j < n_sub; ++j) {
-                // the sub-slot still holds the exponentials of row block i - 2 until the normalise warps have read them
-                ok = __all_sync(0xffffffffu, fused_wait(&bars->slot_free[s][j], (u & 1u) ^ 1u, abort_flag, kSiteGrSlotFree));
+                // the landing slot is free once the exponential warps have taken the scores of row block i - 1 to registers
+                ok = __all_sync(0xffffffffu, fused_wait(&bars->l_free[j], (static_cast<uint32_t>(i) & 1u) ^ 1u, abort_flag, kSiteGrSlotFree));
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 if (lane == 0 && j == 0) ATTNW_STAMP(13, i);
-                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(s * kSlabCols + j * kSub);
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(j * kSub);
                 const uint32_t a_addr = q_addr + static_cast<uint32_t>(s * L::kTileBytes);
                 const uint32_t b_addr = k_addr + static_cast<uint32_t>(j * kSub * 128);  // keys kSub j ... of every atom
                 if (ptx::elect_one()) {
@@ -283,7 +284,7 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         ptx::umma_f16_ss(d_tmem, ptx::umma_desc_kmajor_sw128(a_addr + a_off),
                                          ptx::umma_desc_kmajor_sw128(b_addr + b_off), idesc, k > 0 ? 1u : 0u);
                     }
-                    ptx::umma_commit(&bars->s_full[s][j]);
+                    ptx::umma_commit(&bars->s_full[j]);
                     if (j == n_sub - 1) {
                         ptx::umma_commit(&bars->q_empty[s]);                 // the query tile may be replaced
                         if (last_of_head) ptx::umma_commit(&bars->k_empty);  // ... and the key slab
@@ -292,14 +293,15 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 __syncwarp();
             }
         }
-    } else if (run && warp == kStoreWarpG) {
+    } else if (run && (warp == kStoreWarpG || warp == kStoreWarpG + 1)) {
         // ================= store issuer: one TMA store per filled staging box, in ring order =================
         // Boxes are stored in the order (row block, 64 columns); the boxes of a stream use that stream's ring in turn.
         if (lane == 0) {
             const uint64_t stream_out = ptx::policy_evict_first();
             const uint32_t out_base = ptx::smem_u32(smem + L::kOutOff);
             bool ok = true;
-            for (int i = 0; ok && i < n_items; ++i) {
+            constexpr int kStoreWarps = (kThreads >= 640) ? 2 : 1;  // one store issuer per stream, or one for both
+            for (int i = warp - kStoreWarpG; ok && i < n_items; i += kStoreWarps) {
                 const int gi = begin + i, bh = gi / T, rb = gi % T;
                 const int s = i & 1;
                 const uint32_t ring = s ? L::kRing1 : L::kRing0, base = s ? L::kRing0 : 0;
@@ -328,7 +330,9 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
-        const float c2 = scale_log2e;
+        // never exactly zero, so that a masked score (-3e38) always lands far below the offset; with scale = 0 every
+        // existing score still maps to 2^0
+        const float c2 = fmaxf(scale_log2e, 1.0e-30f);
         const uint64_t c2c2 = ptx::pack2(c2, c2);
         float* mbc_all = reinterpret_cast<float*>(smem + L::kMbcOff);
         float2* part_all = reinterpret_cast<float2*>(smem + L::kPartOff);
@@ -338,40 +342,38 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         for (int i = 0; ok && i < n_items; ++i) {
             const int s = i & 1;
             const uint32_t u = static_cast<uint32_t>(i) >> 1;
-            const uint32_t t_row = t_lane + static_cast<uint32_t>(s * kSlabCols);
             float* mbc = mbc_all + s * kChunksPerBlock * kTile;
             float smax = -3.0e38f, mb = -3.0e38f, l = 0.0f;
             if (stamp) ATTNW_STAMP(0, i);
-            // Every warp waits for the row block's first slot, also one whose boxes lie beyond the last key: a warp
-            // without work must not run ahead of the others and arrive on `posted` for a later row block.
-            ok = __all_sync(0xffffffffu, fused_wait(&bars->s_full[s][0], u & 1u, abort_flag, kSiteGrSFull));
-            if (!ok) break;
-            ptx::tc_fence_after_sync();
-            int cur_slot = 0;
-            if (stamp) ATTNW_STAMP(2, i);
-            // This thread's pieces of the row: the 64-column boxes 2k + par, k = 0, 1.  A whole box is taken at once (64
-            // scores in registers, one offset per box): with two warps per scheduler the dependent chain of a piece
-            // (load, maximum, offset, exponentials, sum, store) has to carry enough independent MUFU work to hide itself.
+            // This thread's pieces of the row: the 64-column boxes 2k + par, k = 0, 1 (landing slot k).  A whole box is taken
+            // at once: 64 scores to registers - the landing slot goes back to the MMA issuer right there -, maximum,
+            // offset, exponentials, sum; the exponentials leave as f16 pairs for the stream's packed region, where they
+            // wait for the row's statistics without holding up the next row block's scores.
 #pragma unroll 1
-            for (int k = 0; k < kSlabCols / kBoxCols / 2; ++k) {
+            for (int k = 0; k < kSubsPerBlock; ++k) {
                 const int bx = 2 * k + par;
                 const int valid = width - bx * kBoxCols;  // columns of this box that exist
-                if (valid <= 0) break;                    // nothing beyond is ever stored (the tensor map clips the box)
-                const int j = (bx * kBoxCols) / kSub;
-                if (j != cur_slot) {
-                    ok = __all_sync(0xffffffffu, fused_wait(&bars->s_full[s][j], u & 1u, abort_flag, kSiteGrSFull));
+                uint32_t r0[kChunk], r1[kChunk];
+                if (k < n_sub) {  // (every warp waits for slot 0, so that a warp without work keeps step)
+                    ok = __all_sync(0xffffffffu, fused_wait(&bars->s_full[k], static_cast<uint32_t>(i) & 1u, abort_flag, kSiteGrSFull));
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
-                    cur_slot = j;
-                    if (stamp && j == 0) ATTNW_STAMP(2, i);
+                    if (stamp && k == 0) ATTNW_STAMP(2, i);
                 }
-                const uint32_t taddr = t_row + static_cast<uint32_t>(bx * kBoxCols);
-                uint32_t r0[kChunk], r1[kChunk];
-                if (stamp) ATTNW_STAMP(16 + 3 * k, i);
-                ptx::tmem_ld_32x32b_x32(taddr, r0);
-                ptx::tmem_ld_32x32b_x32(taddr + kChunk, r1);
-                ptx::tmem_wait_ld();
-                if (stamp) ATTNW_STAMP(17 + 3 * k, i);
+                if (valid <= 0) {  // nothing of the box is ever stored (the tensor map clips it); the slot's barrier counts every warp
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&bars->l_free[k]);
+                    continue;
+                }
+                {
+                    const uint32_t taddr = t_lane + static_cast<uint32_t>(bx * kBoxCols);
+                    ptx::tmem_ld_32x32b_x32(taddr, r0);
+                    ptx::tmem_ld_32x32b_x32(taddr + kChunk, r1);
+                    ptx::tmem_wait_ld();
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&bars->l_free[k]);
+                }
                 if (valid < kBoxCols) {
 #pragma unroll
                     for (int x = 0; x < kChunk; ++x) {
@@ -396,10 +398,11 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 l *= ptx::ex2_approx(mb - mb_new);                   // exactly 1 while the maximum stands
                 mb = mb_new;
                 smax = new_max;
+                uint32_t pk[kChunk];  // the box's 64 exponentials as f16 pairs, in column order
                 {
                     const uint64_t off2 = ptx::pack2(-mb, -mb);
                     uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
-                    const bool ragged = valid < kBoxCols;
+                    // (masked columns hold -3e38 and c2 > 0, so their exponentials are exactly zero)
 #pragma unroll
                     for (int x = 0; x < kChunk; x += 2) {
                         float a0, a1, b0, b1;
@@ -409,16 +412,8 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         a1 = ptx::ex2_approx(a1);
                         b0 = ptx::ex2_approx(b0);
                         b1 = ptx::ex2_approx(b1);
-                        if (ragged) {  // masked columns contribute nothing, also when c2 == 0
-                            a0 = (x + 0 < valid) ? a0 : 0.f;
-                            a1 = (x + 1 < valid) ? a1 : 0.f;
-                            b0 = (x + kChunk + 0 < valid) ? b0 : 0.f;
-                            b1 = (x + kChunk + 1 < valid) ? b1 : 0.f;
-                        }
-                        r0[x] = __float_as_uint(a0);
-                        r0[x + 1] = __float_as_uint(a1);
-                        r1[x] = __float_as_uint(b0);
-                        r1[x + 1] = __float_as_uint(b1);
+                        pk[x >> 1] = ptx::pack_f16x2(a0, a1);
+                        pk[(kChunk >> 1) + (x >> 1)] = ptx::pack_f16x2(b0, b1);
                         acc[(x >> 1) & 1] = ptx::add2(acc[(x >> 1) & 1], ptx::pack2(a0, a1));
                         acc[2 + ((x >> 1) & 1)] = ptx::add2(acc[2 + ((x >> 1) & 1)], ptx::pack2(b0, b1));
                     }
@@ -428,11 +423,13 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     l += (s0 + s1) + (s2 + s3);
                 }
                 if (stamp) ATTNW_STAMP(18 + 3 * k, i);
-                ptx::tmem_st_32x32b_x32(taddr, r0);
-                ptx::tmem_st_32x32b_x32(taddr + kChunk, r1);
+                // the packed region still holds this box of row block i - 2 until its normalise warps have read it
+                ok = __all_sync(0xffffffffu, fused_wait(&bars->pk_free[s][bx], (u & 1u) ^ 1u, abort_flag, kSiteGrSlotFree));
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                ptx::tmem_st_32x32b_x32(t_lane + static_cast<uint32_t>(kPackedCol0 + s * kPackedCols + bx * (kBoxCols / 2)), pk);
                 if (stamp) ATTNW_STAMP(24 + 2 * k, i);
                 mbc[bx * kTile + row] = mb;  // the offset this box's e are relative to
-                if (stamp) ATTNW_STAMP(25 + 2 * k, i);
             }
             if (!ok) break;
             part_all[(s * 2 + par) * kTile + row] = make_float2(mb, l);  // this thread's half of the row
@@ -461,7 +458,6 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         for (int i = first; ok && i < n_items; i += kNormGroups) {
             const int s = i & 1;
             const uint32_t u = static_cast<uint32_t>(i) >> 1;
-            const uint32_t t_row = t_lane + static_cast<uint32_t>(s * kSlabCols);
             const float* mbc = mbc_all + s * kChunksPerBlock * kTile;
             if (stamp) ATTNW_STAMP(10, i);
             // this CTA's exponentials of the row block are in tensor memory and its chunk offsets in shared memory
@@ -559,20 +555,16 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
             for (int b = 0; b < kSlabCols / kBoxCols; ++b) {
                 if (b < n_boxes && ok) {
-                    uint32_t e0[kChunk], e1[kChunk];
-                    const uint32_t taddr = t_row + static_cast<uint32_t>(b * kBoxCols);
-                    ptx::tmem_ld_32x32b_x32(taddr, e0);
-                    ptx::tmem_ld_32x32b_x32(taddr + kChunk, e1);
+                    uint32_t e[kChunk];  // the box's 64 exponentials as f16 pairs
+                    ptx::tmem_ld_32x32b_x32(t_lane + static_cast<uint32_t>(kPackedCol0 + s * kPackedCols + b * (kBoxCols / 2)), e);
                     ptx::tmem_wait_ld();
-                    if ((b + 1) % (kSub / kBoxCols) == 0 || b + 1 == n_boxes) {
-                        // the slot has been read: the scores of row block i + 2 may land in it
-                        ptx::tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(&bars->slot_free[s][b / (kSub / kBoxCols)]);
-                        if (stamp && b / (kSub / kBoxCols) == 0) ATTNW_STAMP(12, i);
-                    }
-                    // staging box of this (row block, 64 columns): ring entry n % kBoxes; the store that last used the
-                    // entry must have read it before anyone overwrites it
+                    // the box has been read: the exponentials of row block i + 2 may take its place
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(&bars->pk_free[s][b]);
+                    if (stamp && b == 0) ATTNW_STAMP(12, i);
+                    // staging box of this (row block, 64 columns): the stream's ring entry m % ring; the store that last
+                    // used the entry must have read it before anyone overwrites it
                     const uint32_t m = u * static_cast<uint32_t>(n_boxes) + static_cast<uint32_t>(b);
                     const uint32_t ring = s ? L::kRing1 : L::kRing0;
                     const uint32_t box = (s ? L::kRing0 : 0) + m % ring, use = m / ring;
@@ -580,36 +572,31 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     if (stamp && b == 1) ATTNW_STAMP(14, i);
                     ok = __all_sync(0xffffffffu, fused_wait(&bars->out_free[box], (use & 1u) ^ 1u, abort_flag, kSiteGrStageFree));
                     if (stamp && b == 1) ATTNW_STAMP(15, i);
-#ifdef ATTNW_GR_NOS2
                     if (ok) {
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(&bars->out_filled[box]);
-                    }
-                    if (false) {
-#else
-                    if (ok) {
-#endif
-                        const uint64_t ff0 = ptx::pack2(f[b], f[b]), ff1 = ff0;
+                        // p = e * f in float32 from f16 operands (one mixed-precision FMA per element unpacks and scales);
+                        // a factor below f16 range rounds to zero, where p < 6e-8 anyway
+                        const uint32_t fh = ptx::pack_f16x2(f[b], f[b]);
 #pragma unroll
                         for (int gg = 0; gg < 8; ++gg) {  // 8 bf16 = one 16-byte piece of the row's 128 bytes
-                            const uint32_t* e = (gg < 4) ? e0 : e1;
-                            const uint64_t ff = (gg < 4) ? ff0 : ff1;
-                            const int x0 = (gg & 3) * 8;
-                            float p[8];
+                            uint32_t w[4];
 #pragma unroll
-                            for (int x = 0; x < 8; x += 2)
-                                ptx::unpack2(ptx::mul2(ptx::pack2(__uint_as_float(e[x0 + x]), __uint_as_float(e[x0 + x + 1])), ff),
-                                             p[x], p[x + 1]);
-                            ptx::st_shared_v4(my_row + ((static_cast<uint32_t>(gg) ^ sw) << 4), ptx::pack_bf16x2(p[0], p[1]),
-                                              ptx::pack_bf16x2(p[2], p[3]), ptx::pack_bf16x2(p[4], p[5]),
-                                              ptx::pack_bf16x2(p[6], p[7]));
+                            for (int x = 0; x < 4; ++x) {
+                                float lo, hi;
+#ifdef ATTNW_GR_CVT_UNPACK
+                                ptx::unpack_f16x2(e[gg * 4 + x], lo, hi);
+                                ptx::unpack2(ptx::mul2(ptx::pack2(lo, hi), ptx::pack2(f[b], f[b])), lo, hi);
+#else
+                                ptx::scale_f16x2(e[gg * 4 + x], fh, lo, hi);
+#endif
+                                w[x] = ptx::pack_bf16x2(lo, hi);
+                            }
+                            ptx::st_shared_v4(my_row + ((static_cast<uint32_t>(gg) ^ sw) << 4), w[0], w[1], w[2], w[3]);
                         }
                         if (stamp && b == 1) ATTNW_STAMP(8, i);
                         ptx::fence_proxy_async_smem();
-                        if (stamp && b == 1) ATTNW_STAMP(9, i);
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(&bars->out_filled[box]);
-                        if (stamp && b == 1) ATTNW_STAMP(5, i);
+                        if (stamp && b == 1) ATTNW_STAMP(9, i);
                     }
                 }
             }

@@ -308,6 +308,23 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
+// {lo, hi} -> packed f16x2 (round to nearest even) and back
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ void unpack_f16x2(uint32_t v, float& lo, float& hi) {
+    asm("{\n\t.reg .f16 l, h;\n\tmov.b32 {l, h}, %2;\n\tcvt.f32.f16 %0, l;\n\tcvt.f32.f16 %1, h;\n\t}" : "=f"(lo), "=f"(hi) : "r"(v));
+}
+// {lo, hi} of a packed f16x2, each times the f16 factor `f16_scale` (low half of the register), as float32:
+// one mixed-precision FMA per element unpacks and scales.
+__device__ __forceinline__ void scale_f16x2(uint32_t v, uint32_t f16_scale, float& lo, float& hi) {
+    asm("{\n\t.reg .f16 l, h, f, g;\n\tmov.b32 {l, h}, %2;\n\tmov.b32 {f, g}, %3;\n\t"
+        "fma.rn.f32.f16 %0, l, f, 0f00000000;\n\tfma.rn.f32.f16 %1, h, f, 0f00000000;\n\t}"
+        : "=f"(lo), "=f"(hi)
+        : "r"(v), "r"(f16_scale));
+}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }

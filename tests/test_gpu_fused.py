@@ -79,6 +79,37 @@ def test_gridrow_variant_matches_oracle(attnw, B, H, N, d):
         assert_close_to_oracle(P, oracle.attnw(q, k, scale), f"gridrow B{B} H{H} N{N} d{d}")
 
 
+def test_gridrow_zero_scale_large_logits_and_identical_keys(attnw):
+    # scale = 0 with masked columns (the last CTA of the group holds 8 of its 256 columns): exactly uniform
+    q, k = small_fused_inputs(1, 2, 264, 64, stream=31)
+    P = run_fused(attnw, q, k, 0.0, torch.bfloat16, variant="gridrow")
+    assert_close_to_oracle(P, oracle.attnw(q, k, 0.0), "gridrow scale 0")
+    # near one-hot rows (sigma = 4): the f16 intermediate of the exponentials must stay inside the bf16 tolerance
+    q, k = small_fused_inputs(1, 2, 2048, 128, sigma=4.0, stream=57)
+    scale = float(np.float32(1.0 / math.sqrt(128.0)))
+    ref = oracle.attnw(q, k, scale)
+    assert ref.max() > 0.9
+    assert_close_to_oracle(run_fused(attnw, q, k, scale, torch.bfloat16, variant="gridrow"), ref, "gridrow sigma 4")
+    # identical keys: exactly uniform after rounding to bf16
+    key = inputs.normal_bf16_bits(3, 3, 128, 1.0)
+    kk = np.broadcast_to(key, (1, 2, 2048, 128)).copy()
+    P = run_fused(attnw, q, kk, 0.3, torch.bfloat16, variant="gridrow")
+    assert bool((P == 1.0 / 2048).all())
+    # beyond its range, or for float32 output, the kernel refuses instead of silently switching
+    big = torch.zeros((1, 1, 4104, 64), dtype=torch.bfloat16, device="cuda")
+    attnw.set_fused_variant("gridrow")
+    try:
+        with pytest.raises(attnw.AttnwError) as e:
+            attnw.attnw_fused(big, big, 0.1)
+        assert e.value.code == 4
+        small = torch.zeros((1, 1, 128, 64), dtype=torch.bfloat16, device="cuda")
+        with pytest.raises(attnw.AttnwError) as e:
+            attnw.attnw_fused(small, small, 0.1, out_dtype=torch.float32)
+        assert e.value.code == 4
+    finally:
+        attnw.set_fused_variant("auto")
+
+
 def test_default_choice_splits_a_call_over_both_kernels(attnw):
     # B*H = 32, N = 2048: 33 clusters of 4 leave 16 SMs idle and walk 16 rounds of row blocks, so the default
     # choice gives two heads to the two-pass kernel on a side stream; the whole of P must be there afterwards
