@@ -18,7 +18,6 @@ from __future__ import annotations
 import argparse
 import json
 import os
-import subprocess
 import sys
 import threading
 import time
@@ -35,13 +34,20 @@ HEADLINE = "c3"
 # Fallback peaks (an earlier measurement on this machine) used only when MEASURED_PEAKS.json is absent.
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures
-# summarised under profiles/; None until a capture exists for that kernel.
-# (c3, default variant: the split launch gives 107 of 128 heads to the resident kernel and 21 to the two-pass
-# kernel; each kernel's capture covers 16 heads, so the launch's traffic is the head-weighted sum.)
-NCU_TRAFFIC_BYTES = {"c3": (107 * (33.66e6 + 476.56e6) + 21 * (33.97e6 + 477.98e6)) / 16,
-                     "c3_resident": 8 * (33.66e6 + 476.56e6), "c3_two_pass": 8 * (33.97e6 + 477.98e6),
-                     "c4": 4 * (268.45e6 + 98.18e6)}
+# Measured traffic per launch comes from profiles/ncu_traffic.json, which every capture summarised under profiles/
+# updates (bytes per head or per row of the reduced case, scaled here by the units one full launch processes).
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+
+
+def measured_traffic(kernel_key: str, units: float):
+    """Bytes one launch moves according to the ncu capture of `kernel_key` (DRAM reads + bytes the SMs wrote towards
+    L2: the DRAM write counter misses what is still dirty in L2 when the kernel ends), or None without a capture."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            entry = json.load(f)[kernel_key]
+        return float(entry["bytes_per_unit"]) * units
+    except Exception:
+        return None
 
 
 def load_peaks():
@@ -160,6 +166,29 @@ def oracle_sample_rate(w, target_seconds: float, seed_offset: int = 0):
     return value, info, dt, n_rows
 
 
+def paper_cpu_rows_line(target_seconds: float = 2.0):
+    """The CPU program of Section VI-A as the paper ran it - C, 32-bit floats, ONE core, caching and recomputing forms
+    - on rows of the row-Softmax configuration c4 (8192 columns), a bounded sample each: the neighbour of the two CPU
+    columns of Table I on this host.  Context beside the oracle line, not a target."""
+    import oracle
+    from paper_2407_13885_b200 import inputs
+    w = inputs.WORKLOADS["c4"]
+    out = {"workload": f"c4 rows: float32 scores [rows x {w.cols}], N(0,{w.sigma:g}^2)", "cores": 1, "kind": "paper_cpu_program",
+           "unit": UNIT}
+    rows = 1024
+    Z = inputs.make_scores(w, 0, rows)
+    for form in ("caching", "recomputing"):
+        reps, dt = 0, 0.0
+        while dt < target_seconds and reps < 64:
+            t0 = time.perf_counter()
+            oracle.paper_cpu_softmax(Z, form)
+            dt += time.perf_counter() - t0
+            reps += 1
+        out[form] = {"value": reps * rows * w.cols / dt, "rows": rows, "passes": reps, "seconds": dt}
+    out["caching_over_recomputing"] = out["caching"]["value"] / out["recomputing"]["value"]
+    return out
+
+
 def run_reference(args):
     rank, world, _ = dist_env()
     if rank != 0:
@@ -190,11 +219,14 @@ def run_reference(args):
     return 0
 
 
-def workload_config(w, world):
+def workload_config(w, world, scaling="weak"):
     cfg = {"workload": f"{w.name}: fused attention weights B={w.B} H={w.H} N={w.N} d={w.d}, Q,K bf16 N(0,{w.sigma:g}^2), "
                        f"scale={w.scale:.9g}, P {w.p_dtype}",
            "B": w.B, "H": w.H, "N": w.N, "d": w.d, "p_dtype": w.p_dtype,
-           "parallelism": f"{world} x independent replicas of the workload (heads are independent; no collective)",
+           "parallelism": (f"{world} x independent replicas of the workload (heads are independent; no collective)"
+                           if scaling == "weak" else
+                           f"the workload's {w.B * w.H} heads dealt out over {world} ranks (quotient + remainder on the first "
+                           "ranks; heads are independent; no collective)"),
            "l2": "no flush: each launch streams 4.56 GB (Q+K 268 MB, P 4.29 GB), far beyond the 126 MB L2"}
     return cfg
 
@@ -386,6 +418,18 @@ def run_profile_case(args):
     return 0
 
 
+def headline_kernel(variant: str, w):
+    """(description, key into profiles/ncu_traffic.json) of the kernel `attnw_fused` runs for this workload."""
+    bf16 = w.p_dtype == "bf16"
+    if variant == "gridrow" or (variant == "auto" and bf16 and w.N <= 4096):
+        return (f"attnw_gridrow_kernel<{w.d}> (groups of {(w.N + 255) // 256} CTAs on a cooperative grid, one launch)",
+                f"attnw_gridrow_d{w.d}_N{w.N}")
+    if variant == "resident" and bf16 and w.N <= 8192:
+        return (f"attnw_resident_kernel<{w.d}> (SRAM-resident, clusters of {(w.N + 511) // 512})",
+                f"attnw_resident_d{w.d}_N{w.N}")
+    return (f"attnw_fused_kernel<{w.d}, {w.p_dtype}> (two-pass)", f"attnw_fused_d{w.d}_N{w.N}")
+
+
 def run_ours(args):
     import torch
     from paper_2407_13885_b200 import binding, inputs  # raises if libattnw.so is missing: no fallback
@@ -404,8 +448,20 @@ def run_ours(args):
     peaks = load_peaks()
     binding.set_fused_variant(args.variant)
 
-    # seeded inputs: every rank draws its own replica of the workload (weak scaling)
-    q, k = inputs.make_qk(w, seed=inputs.SEED + rank)
+    # seeded inputs: every rank draws its own replica of the workload (weak scaling, the default), or its slice of the
+    # heads of ONE workload (--scaling strong); either way no data crosses ranks
+    h_begin, h_end, seed = inputs.rank_heads(w, rank, world, args.scaling)
+    n_heads = h_end - h_begin
+    if n_heads < 1:
+        raise SystemExit(f"rank {rank} owns no head of {w.name}: fewer heads than ranks")
+    q, k = inputs.make_qk(w, h_begin, h_end, seed=seed)
+    if args.scaling == "strong":
+        w_local = inputs.Workload(w.name, "fused", B=1, H=n_heads, N=w.N, d=w.d, sigma=w.sigma, scale=w.scale,
+                                  p_dtype=w.p_dtype, cfg_id=w.cfg_id)
+    else:
+        w_local = w
+    w_total_elements = w.elements if args.scaling == "strong" else world * w.elements
+    w_whole, w = w, w_local
     shape = (w.B, w.H, w.N, w.d)
     Qh = torch.from_numpy(q.view(np.int16)).view(torch.bfloat16).reshape(shape).pin_memory()
     Kh = torch.from_numpy(k.view(np.int16)).view(torch.bfloat16).reshape(shape).pin_memory()
@@ -429,17 +485,19 @@ def run_ours(args):
     sampler = ClockSampler(local)
     sampler.start()
     binding.launch_count(reset=True)
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    start.record()
-    for _ in range(args.steps):
+    # one event after every step (launches stay back to back; nothing synchronises inside the timed region)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    marks[0].record()
+    for i in range(args.steps):
         step()
-    stop.record()
+        marks[i + 1].record()
     torch.cuda.synchronize()
     barrier()
     launches = binding.launch_count()
     sampler.halt.set()
     sampler.join()
-    elapsed_ms = start.elapsed_time(stop)
+    elapsed_ms = marks[0].elapsed_time(marks[-1])
+    per_step = np.array([marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)])
     status = binding.query_status()
     if status != 0:
         raise SystemExit(f"device status word {status:#x}: a bounded wait gave up; timing is invalid")
@@ -452,7 +510,7 @@ def run_ours(args):
         dist.all_reduce(lt, op=dist.ReduceOp.SUM)
         launches = int(lt.item())
     ms_per_step = elapsed_ms / args.steps
-    value = world * w.elements / (ms_per_step * 1e-3)
+    value = w_total_elements / (ms_per_step * 1e-3)
 
     # ---- end to end through the host-buffer C-ABI call ----
     e2e = None
@@ -471,7 +529,7 @@ def run_ours(args):
             t = torch.tensor([dt], dtype=torch.float64, device="cuda")
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             dt = float(t.item())
-        e2e = {"value": world * w.elements * e2e_steps / dt, "unit": UNIT,
+        e2e = {"value": w_total_elements * e2e_steps / dt, "unit": UNIT,
                "h2d_bytes_per_step": w.in_bytes, "d2h_bytes_per_step": w.p_bytes,
                "steps": e2e_steps, "ms_per_step": 1e3 * dt / e2e_steps,
                "note": "attnw_fused_host: pinned host Q,K -> device, kernel, P -> pinned host, pipelined over "
@@ -487,24 +545,27 @@ def run_ours(args):
     achieved = bytes_alg / kernel_s / 1e9
     t_hbm = bytes_alg / (peaks["hbm_gbs"] * 1e9)
     t_flop = w.flops / (peaks["bf16_tflops"] * 1e12)
+    kernel_name, kernel_key = headline_kernel(args.variant, w)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"],
-                "traffic": NCU_TRAFFIC_BYTES.get(w.name + {"two_pass": "_two_pass", "resident": "_resident"}.get(args.variant, "")),
+                "traffic": measured_traffic(kernel_key, w.B * w.H),
+                "traffic_source": f"profiles/ncu_traffic.json[{kernel_key}] x {w.B * w.H} heads",
                 "peak_source": f"of {peaks['source']}",
                 "algorithmic_bytes_per_launch": bytes_alg,
                 "roofline_time_us": 1e6 * max(t_hbm, t_flop), "kernel_time_us": 1e6 * kernel_s,
                 "time_frac_of_roofline": max(t_hbm, t_flop) / kernel_s,
                 "tensor_time_us_at_burst_peak": 1e6 * t_flop,
-                "kernel": "attnw_fused_kernel<128, bf16> (two-pass)" if (args.variant == "two_pass" or w.N > 4096)
-                else ("attnw_resident_kernel<128> (SRAM-resident, clusters of %d)" % ((w.N + 511) // 512)
-                      + (" on the SMs clusters can occupy + attnw_fused_kernel<128, bf16> on the rest: one split launch per step"
-                         if args.variant == "auto" else ""))}
+                "kernel": kernel_name}
+    step_ms = {"median": float(np.median(per_step)), "min": float(per_step.min()), "max": float(per_step.max()),
+               "mean": float(per_step.mean()),
+               "note": "one CUDA event after every launch of the timed region (rank 0); launches back to back"}
+    roofline["frac_at_median_step"] = bytes_alg / (step_ms["median"] * 1e-3) / 1e9 / peaks["hbm_gbs"]
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": workload_config(w, world), "clocks": sampler.summary(), "e2e": e2e,
-            "gpu_launches": launches, "roofline": roofline}
+            "scaling": args.scaling, "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_config(w_whole, world, args.scaling), "clocks": sampler.summary(), "e2e": e2e,
+            "gpu_launches": launches, "roofline": roofline, "step_ms": step_ms}
 
     if not args.no_sustained and world == 1:
         # A multi-second loop of the same launch: the chip settles at its power limit (about 1.45-1.55 GHz
@@ -524,13 +585,17 @@ def run_ours(args):
                              "roofline_frac": bytes_alg / (ms_loop * 1e-3) / 1e9 / peaks["hbm_gbs"],
                              "launches": n_loop,
                              "note": "last 100 of a %.0f s back-to-back loop; power-capped clocks" % args.sustained_seconds}
+        roofline["frac_sustained"] = line["sustained"]["roofline_frac"]
     if not args.no_cpu_baseline:
         _, info, _, _ = oracle_sample_rate(w, args.cpu_seconds)
+        info["paper_cpu_c4"] = paper_cpu_rows_line()
         line["cpu_baseline"] = info
     if not args.no_secondary and world == 1:
         del P, Q, K
         torch.cuda.empty_cache()
         line["reference_streams"] = reference_streams()
+        # the same launch against the write-only stream measured in this run (P is 94 % of the bytes and all writes)
+        roofline["frac_of_write_only_stream"] = achieved / line["reference_streams"]["write_only_gbs"]
         torch.cuda.empty_cache()
         other = {}
         for name in ("c4", "c5", "c2"):
@@ -552,6 +617,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default=HEADLINE, choices=["c2", "c3", "c5"])
+    ap.add_argument("--scaling", choices=["weak", "strong"], default="weak",
+                    help="weak: every rank runs a whole replica (default); strong: the heads of ONE workload are dealt out")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-e2e", action="store_true")

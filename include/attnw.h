@@ -103,12 +103,10 @@ int attnw_set_attn_variant(int variant);
 
 /*
  * Which kernel attnw_fused uses (process-wide; the results are the same within the stated tolerances):
- *   0  choose by shape (default): the SRAM-resident kernel when P is bfloat16 and N <= 4096; the
- *      two-pass kernel otherwise (and always for attnw_fused_f32).  Clusters cannot occupy every SM
- *      (clusters of 8: 120 of 148), so a large call is
- *      split: most heads go to the resident kernel on `stream`, the rest to the two-pass kernel on a
- *      per-device side stream that forks from and joins `stream` with events (first use creates the
- *      side stream and two events); work enqueued on `stream` afterwards sees the whole result.
+ *   0  choose by shape (default): the grid-row kernel (see 4) when P is bfloat16 and N <= 4096; the two-pass
+ *      kernel otherwise (and always for attnw_fused_f32).  On a device that cannot hold a whole group of the
+ *      grid-row kernel at once the older choice applies: the SRAM-resident cluster kernel, with a large call split
+ *      between it and the two-pass kernel on a per-device side stream that forks from and joins `stream` with events.
  *   1  two-pass kernel: statistics pass + normalise pass that recomputes the score tiles; any N
  *   2  SRAM-resident kernel: a cluster of ceil(N/512) <= 16 CTAs keeps a 128-row block of scores in tensor
  *      memory and exchanges local row maxima and sums across CTAs, as the fused kernel of Section VII

@@ -339,6 +339,9 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const bool stamp = warp == 0 && lane == 0;
         (void)stamp;
         bool ok = true;
+#ifdef ATTNW_GR_STAGGER
+        if (par == 1) __nanosleep(ATTNW_GR_STAGGER);
+#endif
         for (int i = 0; ok && i < n_items; ++i) {
             const int s = i & 1;
             const uint32_t u = static_cast<uint32_t>(i) >> 1;
@@ -360,6 +363,7 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     ptx::tc_fence_after_sync();
                     if (stamp && k == 0) ATTNW_STAMP(2, i);
                 }
+                if (stamp) ATTNW_STAMP(17 + 3 * k, i);
                 if (valid <= 0) {  // nothing of the box is ever stored (the tensor map clips it); the slot's barrier counts every warp
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(&bars->l_free[k]);
@@ -398,6 +402,7 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 l *= ptx::ex2_approx(mb - mb_new);                   // exactly 1 while the maximum stands
                 mb = mb_new;
                 smax = new_max;
+                if (stamp) ATTNW_STAMP(16 + 3 * k, i);
                 uint32_t pk[kChunk];  // the box's 64 exponentials as f16 pairs, in column order
                 {
                     const uint64_t off2 = ptx::pack2(-mb, -mb);
@@ -406,8 +411,10 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
                     for (int x = 0; x < kChunk; x += 2) {
                         float a0, a1, b0, b1;
-                        ptx::unpack2(ptx::fma2(ptx::pack2(__uint_as_float(r0[x]), __uint_as_float(r0[x + 1])), c2c2, off2), a0, a1);
-                        ptx::unpack2(ptx::fma2(ptx::pack2(__uint_as_float(r1[x]), __uint_as_float(r1[x + 1])), c2c2, off2), b0, b1);
+                        const uint64_t xa = ptx::fma2(ptx::pack2(__uint_as_float(r0[x]), __uint_as_float(r0[x + 1])), c2c2, off2);
+                        const uint64_t xb = ptx::fma2(ptx::pack2(__uint_as_float(r1[x]), __uint_as_float(r1[x + 1])), c2c2, off2);
+                        ptx::unpack2(xa, a0, a1);
+                        ptx::unpack2(xb, b0, b1);
                         a0 = ptx::ex2_approx(a0);
                         a1 = ptx::ex2_approx(a1);
                         b0 = ptx::ex2_approx(b0);
@@ -569,9 +576,9 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const uint32_t ring = s ? L::kRing1 : L::kRing0;
                     const uint32_t box = (s ? L::kRing0 : 0) + m % ring, use = m / ring;
                     const uint32_t my_row = out_base + box * kBoxBytes + static_cast<uint32_t>(row * 128);
-                    if (stamp && b == 1) ATTNW_STAMP(14, i);
+                    if (stamp && b == 2) ATTNW_STAMP(14, i);
                     ok = __all_sync(0xffffffffu, fused_wait(&bars->out_free[box], (use & 1u) ^ 1u, abort_flag, kSiteGrStageFree));
-                    if (stamp && b == 1) ATTNW_STAMP(15, i);
+                    if (stamp && b == 2) ATTNW_STAMP(15, i);
                     if (ok) {
                         // p = e * f in float32 from f16 operands (one mixed-precision FMA per element unpacks and scales);
                         // a factor below f16 range rounds to zero, where p < 6e-8 anyway
@@ -592,11 +599,11 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             }
                             ptx::st_shared_v4(my_row + ((static_cast<uint32_t>(gg) ^ sw) << 4), w[0], w[1], w[2], w[3]);
                         }
-                        if (stamp && b == 1) ATTNW_STAMP(8, i);
+                        if (stamp && b == 2) ATTNW_STAMP(8, i);
                         ptx::fence_proxy_async_smem();
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(&bars->out_filled[box]);
-                        if (stamp && b == 1) ATTNW_STAMP(9, i);
+                        if (stamp && b == 2) ATTNW_STAMP(9, i);
                     }
                 }
             }

@@ -177,3 +177,18 @@ def shard_range(total: int, rank: int, world: int) -> tuple[int, int]:
     q, r = divmod(total, world)
     begin = rank * q + min(rank, r)
     return begin, begin + q + (1 if rank < r else 0)
+
+
+def rank_heads(w: Workload, rank: int, world: int, scaling: str = "weak") -> tuple[int, int, int]:
+    """Heads ``[begin, end)`` (flattened b*H + h) a rank computes, and the seed it draws them with.
+
+    ``weak``: every rank owns a whole replica of the workload, drawn with its own seed (per-GPU work fixed).
+    ``strong``: ONE workload; its heads are dealt out with :func:`shard_range` (quotient plus one extra head on the
+    first ranks), every rank draws only its slice with the common seed, and no data crosses ranks: a head's rows
+    need nothing from another head (Section VI-B's partition; Section VIII's "multiple cards")."""
+    if scaling == "weak":
+        return 0, w.B * w.H, SEED + rank
+    if scaling == "strong":
+        begin, end = shard_range(w.B * w.H, rank, world)
+        return begin, end, SEED
+    raise ValueError("scaling must be 'weak' or 'strong'")

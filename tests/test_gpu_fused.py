@@ -110,15 +110,14 @@ def test_gridrow_zero_scale_large_logits_and_identical_keys(attnw):
         attnw.set_fused_variant("auto")
 
 
-def test_default_choice_splits_a_call_over_both_kernels(attnw):
-    # B*H = 32, N = 2048: 33 clusters of 4 leave 16 SMs idle and walk 16 rounds of row blocks, so the default
-    # choice gives two heads to the two-pass kernel on a side stream; the whole of P must be there afterwards
+def test_default_choice_for_bf16_up_to_4096_is_one_gridrow_launch(attnw):
+    # B*H = 32, N = 2048: the default serves the whole call with one cooperative launch of the grid-row kernel
     q, k = small_fused_inputs(4, 8, 2048, 64, stream=99)
     scale = float(np.float32(0.125))
     attnw.launch_count(reset=True)
     P = run_fused(attnw, q, k, scale, torch.bfloat16, variant="auto")
-    assert attnw.launch_count() == 2
-    assert_close_to_oracle(P, oracle.attnw(q, k, scale), "split launch B4 H8 N2048 d64")
+    assert attnw.launch_count() == 1
+    assert_close_to_oracle(P, oracle.attnw(q, k, scale), "default launch B4 H8 N2048 d64")
 
 
 def test_resident_variant_large_logits_and_limits(attnw):
