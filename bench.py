@@ -630,7 +630,12 @@ def main():
                     help="kernel behind attnw_fused (see attnw_set_fused_variant)")
     ap.add_argument("--profile", choices=["fused", "rows", "rows_long", "attention", "project"], default=None,
                     help="run a reduced case of one kernel for an ncu capture instead of the benchmark")
+    ap.add_argument("--timeline", action="store_true",
+                    help="per-phase cycle table of the headline kernel from an instrumented build (see timeline.py)")
     args = ap.parse_args()
+    if args.timeline:
+        from paper_2407_13885_b200 import timeline
+        return timeline.main([])
     if args.impl == "reference":
         return run_reference(args)
     if args.profile:

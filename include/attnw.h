@@ -16,7 +16,8 @@
  *   - `stream` is a cudaStream_t (NULL = the legacy default stream).  Calls enqueue work and
  *     return; they do not synchronise.
  *   - The return value is an attnw_status.  Argument errors are detected on the host and
- *     nothing is launched.  ATTNW_ERR_TIMEOUT is only ever reported by attnw_query_status().
+ *     nothing is launched.  ATTNW_ERR_TIMEOUT is reported by attnw_query_status() and by the *_host calls (which
+ *     synchronise anyway); the asynchronous device entry points cannot know of it when they return.
  *   - Inputs must be finite.  Non-finite inputs give unspecified values in the rows they
  *     touch and never a fault.
  *   - Runs on the current CUDA device, which must be compute capability 10.x.  There is no
@@ -60,7 +61,7 @@ int attnw_fused_f32(const void* Q, const void* K, void* P, int B, int H, int N, 
 
 /*
  * attn_fused: O[b,h,i,c] = sum_j P[b,h,i,j] * V[b,h,j,c] with P as defined for attnw_fused - Attention(Q, K, V) of
- * Section IV, the product with V that Section IX leaves as future work - in one kernel; neither the scores nor the
+ * Section IV, the product with V that Section VIII leaves as future work - in one kernel; neither the scores nor the
  * weights reach HBM.
  *
  *   Q, K, V  device, bfloat16, [B, H, N, d]                    (read only)
@@ -74,7 +75,7 @@ int attn_fused(const void* Q, const void* K, const void* V, void* O, int B, int 
 
 /*
  * attnw_project_qk: the linear transformation of the inputs into queries and keys in front of the attention weights
- * (Section IV; a step the paper leaves to the vendor's matmul and names as future work in Section IX), for all heads in
+ * (Section IV; a step the paper leaves to the vendor's matmul and names as future work in Section VIII), for all heads in
  * one launch:   Q[b,h,n,c] = sum_m X[b,n,m] * Wq[h,c,m],   K[b,h,n,c] = sum_m X[b,n,m] * Wk[h,c,m].
  *
  *   X        device, bfloat16, [B, N, d_model]                  (read only)
@@ -112,7 +113,7 @@ int attnw_set_attn_variant(int variant);
  *      memory and exchanges local row maxima and sums across CTAs, as the fused kernel of Section VII
  *      does across Tensix cores; serves bfloat16 P and N <= 8192, any other call then returns
  *      ATTNW_ERR_UNSUPPORTED
- *   3  the same kernel with the exchange the paper leaves as future work (Section IX): the rows are dealt out to
+ *   3  the same kernel with the exchange the paper leaves as future work (Section VIII): the rows are dealt out to
  *      the CTAs of the cluster, the owner of a row receives its local maxima and sums, reduces them once and
  *      sends the global values to every CTA (reduce and broadcast) instead of every CTA reducing redundantly
  *   4  grid-row kernel: the SRAM-resident design on a cooperative grid of one CTA per SM.  Consecutive ceil(N/256)
@@ -172,13 +173,27 @@ int softmax_rows_host(const void* S, void* P, long long rows, long long cols, in
 int attnw_host_release(void);
 
 /*
- * Device-side failure reporting.  Every wait inside the kernels is bounded; a wait that gives
- * up records a code in a per-device status word, makes the kernel unwind and return normally,
- * and the output of that launch is then undefined.  attnw_query_status() synchronises
- * `stream`, stores the word in *device_status (0 = no failure; otherwise an implementation
- * code naming the wait that gave up), clears it, and returns ATTNW_OK or ATTNW_ERR_TIMEOUT.
+ * Device-side failure reporting.  Every wait inside the kernels is bounded (about one second); a wait that gives
+ * up records a code in a per-device status word, makes the kernel unwind and return normally, and the output of
+ * that launch is then undefined.
+ * The word is STICKY: while it is non-zero, every later launch of the tensor-core kernels (attnw_fused*, attn_fused,
+ * attnw_project_qk) and of the shared-memory tier of softmax_rows* returns at once WITHOUT WRITING ITS OUTPUT - the
+ * call itself still returns ATTNW_OK, since it only enqueues - so that no work piles up behind a device that has
+ * stopped making progress.  The register and streaming tiers of softmax_rows* have no waits and ignore the word.
+ * attnw_query_status() synchronises `stream`, stores the word in *device_status (0 = no failure; otherwise
+ * 0x80000000 | an implementation code naming the wait that gave up), clears it, and returns ATTNW_OK or
+ * ATTNW_ERR_TIMEOUT; after it has returned ATTNW_ERR_TIMEOUT, launches work again.  attnw_fused_host and
+ * softmax_rows_host read and clear the word themselves before they return.
  */
 int attnw_query_status(void* stream, unsigned int* device_status);
+
+/*
+ * Self-test of the failure path (the paper has no counterpart): launches one warp that waits, for at most
+ * `limit_cycles` SM clocks (1 ... 2e9), on a barrier nobody arrives on, gives up, records site code 127 in the status
+ * word and returns.  Nothing else is touched and no kernel of the library is altered; afterwards the device is in the
+ * sticky state described above until attnw_query_status() is called.  ATTNW_ERR_BAD_SHAPE if the limit is out of range.
+ */
+int attnw_selftest_wait_timeout(long long limit_cycles, void* stream);
 
 /* Number of kernels this library has launched in the calling process since load / last reset
  * (reset = 1 returns the count and then sets it to zero). */

@@ -27,6 +27,7 @@ SIGNATURES = {
     "softmax_rows_host": (_int, [_vp, _vp, _ll, _ll, _int]),
     "attnw_host_release": (_int, []),
     "attnw_query_status": (_int, [_vp, ctypes.POINTER(ctypes.c_uint)]),
+    "attnw_selftest_wait_timeout": (_int, [_ll, _vp]),
     "attnw_set_fused_variant": (_int, [_int]),
     "attnw_set_attn_variant": (_int, [_int]),
     "attnw_set_rows_variant": (_int, [_int]),
@@ -255,3 +256,9 @@ def query_status(stream=None) -> int:
     if code not in (0, 6):
         raise AttnwError(code, "attnw_query_status")
     return int(word.value)
+
+
+def selftest_wait_timeout(limit_cycles: int = 1_000_000, stream=None) -> None:
+    """Launches the failure-path self-test: one warp waits ``limit_cycles`` SM clocks on a barrier nobody arrives on,
+    gives up and records site 127 in the device status word (see ``attnw_selftest_wait_timeout``)."""
+    _check(lib.attnw_selftest_wait_timeout(int(limit_cycles), _stream_ptr(stream)), "attnw_selftest_wait_timeout")

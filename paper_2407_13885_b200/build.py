@@ -20,13 +20,12 @@ def nvcc_path() -> str:
     raise RuntimeError("nvcc not found; it is needed to build libattnw.so")
 
 
-def nvcc_command(out: str, verbose_ptxas: bool = False) -> list[str]:
+def nvcc_command(out: str, verbose_ptxas: bool = False, defines: tuple[str, ...] = ()) -> list[str]:
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-o", out, *SOURCES]
     if verbose_ptxas:
         cmd[1:1] = ["-Xptxas", "-v"]
-    # Extra -D definitions for experiments and debug builds, e.g. ATTNW_DEFINES="ATTNW_TIMELINE=700".
-    for d in os.environ.get("ATTNW_DEFINES", "").split():
+    for d in defines:
         cmd.insert(1, "-D" + d)
     return cmd
 
@@ -38,18 +37,23 @@ def is_stale() -> bool:
     return any(os.path.getmtime(d) > built for d in _DEPS)
 
 
-def build_library(force: bool = False, verbose_ptxas: bool = False) -> str:
-    """Compile if the library is missing or older than its sources; returns its path."""
-    if not force and not is_stale():
+def build_library(force: bool = False, verbose_ptxas: bool = False, defines: tuple[str, ...] = (),
+                  out: str | None = None) -> str:
+    """Compile if the library is missing or older than its sources; returns its path.  `defines` and `out` build a
+    variant beside the product library (the instrumented build of timeline.py); the product library has none."""
+    target = out or LIB_PATH
+    if defines and out is None:
+        raise ValueError("a build with extra definitions needs its own output path")
+    if not force and out is None and not is_stale():
         return LIB_PATH
-    tmp = LIB_PATH + f".tmp{os.getpid()}"
-    proc = subprocess.run(nvcc_command(tmp, verbose_ptxas), capture_output=True, text=True)
+    tmp = target + f".tmp{os.getpid()}"
+    proc = subprocess.run(nvcc_command(tmp, verbose_ptxas, defines), capture_output=True, text=True)
     if proc.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + proc.stdout + proc.stderr)
-    os.replace(tmp, LIB_PATH)
+    os.replace(tmp, target)
     if verbose_ptxas:
         print(proc.stderr)
-    return LIB_PATH
+    return target
 
 
 if __name__ == "__main__":

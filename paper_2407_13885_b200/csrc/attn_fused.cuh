@@ -1,5 +1,5 @@
 // Fused attention O = Softmax(scale * Q K^T) V for sm_100a: Attention(Q, K, V) of Section IV, the product with V
-// that the paper leaves as future work (Section IX), without ever writing the attention weights to HBM.
+// that the paper leaves as future work (Section VIII), without ever writing the attention weights to HBM.
 //
 // The structure is the two-pass kernel of attnw_fused.cuh: a CTA owns 256 query rows (two tiles that share every
 // key tile); pass 1 streams the key tiles and keeps, per row, the running maximum and the sum of exponentials

@@ -1,5 +1,5 @@
 // Fused attention O = Softmax(scale * Q K^T) V for sm_100a in ONE pass over the keys: Attention(Q, K, V) of
-// Section IV (the product with V is the paper's future work, Section IX) with the online form of Eq. 1.
+// Section IV (the product with V is the paper's future work, Section VIII) with the online form of Eq. 1.
 //
 // A CTA owns 256 query rows (two tiles).  Per key tile j and query tile q:
 //   MMA 1     S = Q_q K_j^T                       128 x 128 fp32 in tensor memory (one buffer per query tile)

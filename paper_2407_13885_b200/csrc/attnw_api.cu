@@ -26,6 +26,37 @@ namespace {
 using namespace attnw;
 
 constexpr int kMaxDevices = 64;
+constexpr uint32_t kSiteSelfTest = 127;  // wait site of attnw_selftest_wait_timeout (low byte of the status word)
+
+// Not part of any product path: one thread waits, with the caller's limit, on an mbarrier that nobody arrives on,
+// gives up, records the site in the per-device status word and returns - the unwinding every kernel's bounded wait
+// follows, made reachable for a test without touching the waits of the real kernels.
+__global__ void wait_timeout_selftest_kernel(long long limit_cycles) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        ptx::mbar_fence_init();
+        const long long t0 = clock64();
+        while (!ptx::mbar_try_wait(&bar, 0u)) {
+            if (clock64() - t0 > limit_cycles) {
+                atomicCAS(&g_attnw_status, 0u, 0x80000000u | kSiteSelfTest);
+                break;
+            }
+        }
+    }
+}
+
+// Reads the current device's status word after the caller has synchronised; a recorded failure is cleared and
+// reported once.
+int read_and_clear_status(unsigned int* word_out) {
+    unsigned int word = 0;
+    if (cudaMemcpyFromSymbol(&word, attnw::g_attnw_status, sizeof(word)) != cudaSuccess) return ATTNW_ERR_CUDA;
+    if (word_out) *word_out = word;
+    if (word == 0) return ATTNW_OK;
+    const unsigned int zero = 0;
+    if (cudaMemcpyToSymbol(attnw::g_attnw_status, &zero, sizeof(zero)) != cudaSuccess) return ATTNW_ERR_CUDA;
+    return ATTNW_ERR_TIMEOUT;
+}
 constexpr int kVersion = 100;  // 0.1.0
 
 std::atomic<long long> g_launches{0};
@@ -768,6 +799,8 @@ int attnw_fused_host(const void* Q, const void* K, void* P, int B, int H, int N,
     if (d != 64 && d != 128) return ATTNW_ERR_UNSUPPORTED;
     const long long bh = static_cast<long long>(B) * H;
     if (bh > INT_MAX || N > (1 << 24)) return ATTNW_ERR_BAD_SHAPE;
+    if (!(scale >= 0.0f) || !std::isfinite(scale)) return ATTNW_ERR_BAD_SHAPE;
+    if ((static_cast<unsigned long long>(N) * esize) % 16 != 0) return ATTNW_ERR_MISALIGNED;  // before anything is queued
     HostStaging* st = nullptr;
     int rc = staging_for_current_device(&st);
     if (rc != ATTNW_OK) return rc;
@@ -791,19 +824,25 @@ int attnw_fused_host(const void* Q, const void* K, void* P, int B, int H, int N,
         const int slot = piece & 1;
         cudaStream_t s = st->stream[slot];
         if (cudaMemcpyAsync(st->buf[slot][0], q + h0 * qk_head, g * qk_head, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-            cudaMemcpyAsync(st->buf[slot][1], k + h0 * qk_head, g * qk_head, cudaMemcpyHostToDevice, s) != cudaSuccess)
-            return ATTNW_ERR_CUDA;
+            cudaMemcpyAsync(st->buf[slot][1], k + h0 * qk_head, g * qk_head, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+            rc = ATTNW_ERR_CUDA;
+            break;
+        }
         rc = p_is_f32 ? attnw_fused_f32(st->buf[slot][0], st->buf[slot][1], st->buf[slot][2], 1, static_cast<int>(g), N,
                                         d, scale, s)
                       : attnw_fused(st->buf[slot][0], st->buf[slot][1], st->buf[slot][2], 1, static_cast<int>(g), N, d,
                                     scale, s);
-        if (rc != ATTNW_OK) return rc;
-        if (cudaMemcpyAsync(p + h0 * p_head, st->buf[slot][2], g * p_head, cudaMemcpyDeviceToHost, s) != cudaSuccess)
-            return ATTNW_ERR_CUDA;
+        if (rc != ATTNW_OK) break;
+        if (cudaMemcpyAsync(p + h0 * p_head, st->buf[slot][2], g * p_head, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+            rc = ATTNW_ERR_CUDA;
+            break;
+        }
     }
+    // On every path, also after an error: no copy may still be reading or writing the caller's buffers on return.
     for (int slot = 0; slot < 2; ++slot)
-        if (cudaStreamSynchronize(st->stream[slot]) != cudaSuccess) return ATTNW_ERR_CUDA;
-    return ATTNW_OK;
+        if (cudaStreamSynchronize(st->stream[slot]) != cudaSuccess && rc == ATTNW_OK) rc = ATTNW_ERR_CUDA;
+    if (rc != ATTNW_OK) return rc;
+    return read_and_clear_status(nullptr);  // a wait that gave up inside a kernel: the result is not valid
 }
 
 int softmax_rows_host(const void* S, void* P, long long rows, long long cols, int p_is_f32) {
@@ -831,18 +870,24 @@ int softmax_rows_host(const void* S, void* P, long long rows, long long cols, in
         const int slot = piece & 1;
         cudaStream_t s = st->stream[slot];
         if (cudaMemcpyAsync(st->buf[slot][0], src + r0 * cols * 4, static_cast<size_t>(g) * cols * 4,
-                            cudaMemcpyHostToDevice, s) != cudaSuccess)
-            return ATTNW_ERR_CUDA;
+                            cudaMemcpyHostToDevice, s) != cudaSuccess) {
+            rc = ATTNW_ERR_CUDA;
+            break;
+        }
         rc = p_is_f32 ? softmax_rows_f32(st->buf[slot][0], st->buf[slot][2], g, cols, s)
                       : softmax_rows(st->buf[slot][0], st->buf[slot][2], g, cols, s);
-        if (rc != ATTNW_OK) return rc;
+        if (rc != ATTNW_OK) break;
         if (cudaMemcpyAsync(dst + r0 * cols * esize, st->buf[slot][2], static_cast<size_t>(g) * cols * esize,
-                            cudaMemcpyDeviceToHost, s) != cudaSuccess)
-            return ATTNW_ERR_CUDA;
+                            cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+            rc = ATTNW_ERR_CUDA;
+            break;
+        }
     }
+    // On every path, also after an error: no copy may still be reading or writing the caller's buffers on return.
     for (int slot = 0; slot < 2; ++slot)
-        if (cudaStreamSynchronize(st->stream[slot]) != cudaSuccess) return ATTNW_ERR_CUDA;
-    return ATTNW_OK;
+        if (cudaStreamSynchronize(st->stream[slot]) != cudaSuccess && rc == ATTNW_OK) rc = ATTNW_ERR_CUDA;
+    if (rc != ATTNW_OK) return rc;
+    return read_and_clear_status(nullptr);  // a wait that gave up inside a kernel: the result is not valid
 }
 
 int attnw_host_release(void) {
@@ -863,13 +908,18 @@ int attnw_host_release(void) {
 int attnw_query_status(void* stream, unsigned int* device_status) {
     if (!device_status) return ATTNW_ERR_NULL_POINTER;
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return ATTNW_ERR_CUDA;
-    unsigned int word = 0;
-    if (cudaMemcpyFromSymbol(&word, attnw::g_attnw_status, sizeof(word)) != cudaSuccess) return ATTNW_ERR_CUDA;
-    *device_status = word;
-    if (word == 0) return ATTNW_OK;
-    const unsigned int zero = 0;
-    if (cudaMemcpyToSymbol(attnw::g_attnw_status, &zero, sizeof(zero)) != cudaSuccess) return ATTNW_ERR_CUDA;
-    return ATTNW_ERR_TIMEOUT;
+    return read_and_clear_status(device_status);
+}
+
+int attnw_selftest_wait_timeout(long long limit_cycles, void* stream) {
+    if (limit_cycles < 1 || limit_cycles > 2000000000ll) return ATTNW_ERR_BAD_SHAPE;  // at most about one second
+    DeviceInfo* dev = nullptr;
+    int rc = current_device(&dev);
+    if (rc != ATTNW_OK) return rc;
+    wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(limit_cycles);
+    if (cudaGetLastError() != cudaSuccess) return ATTNW_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTNW_OK;
 }
 
 int attnw_set_fused_variant(int variant) {
@@ -897,19 +947,7 @@ const char* attnw_strerror(int code) {
 }
 
 int attnw_version(void) { return kVersion; }
-#ifdef ATTNW_CTA_CLOCK
-// Debug builds only (-DATTNW_CTA_CLOCK): per-CTA cycle and nanosecond spans of the last fused launch.
-int attnw_debug_cta_clock(long long* out) {
-    if (cudaDeviceSynchronize() != cudaSuccess) return ATTNW_ERR_CUDA;
-    return cudaMemcpyFromSymbol(out, attnw::g_attnw_cta_clock, sizeof(long long) * 4096 * 4) == cudaSuccess ? ATTNW_OK
-                                                                                                           : ATTNW_ERR_CUDA;
-}
-#endif
 #ifdef ATTNW_TIMELINE
-int attnw_debug_gt(unsigned long long* out) {
-    if (cudaDeviceSynchronize() != cudaSuccess) return ATTNW_ERR_CUDA;
-    return cudaMemcpyFromSymbol(out, attnw::gr::g_attnw_gt, sizeof(unsigned long long) * 160 * 3 * 160) == cudaSuccess ? ATTNW_OK : ATTNW_ERR_CUDA;
-}
 // Debug builds only (-DATTNW_TIMELINE=<cta index>): copies the cycle stamps of that CTA to the host.
 int attnw_debug_timeline(long long* out) {
     if (cudaDeviceSynchronize() != cudaSuccess) return ATTNW_ERR_CUDA;

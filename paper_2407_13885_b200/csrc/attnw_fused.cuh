@@ -38,9 +38,6 @@ __device__ unsigned int g_attnw_status = 0;
 
 // Optional per-role cycle stamps of one CTA (the analogue of the paper's per-operation runtime
 // figures).  Compiled in only with -DATTNW_TIMELINE; the product build has none of it.
-#ifdef ATTNW_CTA_CLOCK
-__device__ long long g_attnw_cta_clock[4096][4];  // per CTA: cycles, nanoseconds, SM id, start ns
-#endif
 #ifdef ATTNW_TIMELINE
 __device__ long long g_attnw_timeline[32][160];
 #define ATTNW_STAMP(ev, it)                                                                       \
@@ -224,13 +221,6 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     FusedBarriers* bars = reinterpret_cast<FusedBarriers*>(smem + L::kBarOff);
     volatile uint32_t* abort_flag = &bars->abort_flag;
 
-#ifdef ATTNW_CTA_CLOCK
-    long long cc0 = 0, ns0 = 0;
-    if (threadIdx.x == 0) {
-        cc0 = clock64();
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns0));
-    }
-#endif
     if (threadIdx.x == 0) bars->prior_failure = *reinterpret_cast<volatile unsigned int*>(&g_attnw_status);
     __syncthreads();
     if (bars->prior_failure != 0u) {  // an earlier CTA gave up: do not queue more waits behind it
@@ -314,14 +304,6 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const int s = it % L::kStages;
                 const uint32_t n = static_cast<uint32_t>(it / L::kStages);
                 if (!fused_wait(&bars->k_empty[s], (n & 1u) ^ 1u, abort_flag, kSiteProducerEmpty)) break;
-                ATTNW_STAMP(0, it);
-#ifdef ATTNW_TIMELINE
-                if (blockIdx.x == ATTNW_TIMELINE && it < 160) {
-                    long long ns;
-                    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
-                    g_attnw_timeline[10][it] = ns;   // wall-clock twin of stamp 0: gives the SM clock under load
-                }
-#endif
                 ptx::mbar_expect_tx(&bars->k_full[s], static_cast<uint32_t>(L::kTileBytes));
                 const int kt = kt0 + (it < T ? it : it - T);
                 for (int a = 0; a < L::kAtoms; ++a)
@@ -356,10 +338,8 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         for (int it = 0; ok && it < total_iters; ++it) {
             const int s = it % L::kStages;
             const uint32_t n = static_cast<uint32_t>(it / L::kStages);
-            if (lane == 0) ATTNW_STAMP(1, it);
             ok = __all_sync(0xffffffffu, fused_wait(&bars->k_full[s], n & 1u, abort_flag, kSiteMmaKFull));
             if (!ok) break;
-            if (lane == 0) ATTNW_STAMP(2, it);
             const int buf = it & 1;
             const uint32_t use = static_cast<uint32_t>(it >> 1);
             const uint32_t b_addr = k_addr + static_cast<uint32_t>(s * L::kTileBytes);
@@ -369,7 +349,6 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 ok = __all_sync(0xffffffffu, fused_wait(&bars->s_empty[q][buf], (use & 1u) ^ 1u, abort_flag,
                                                         kSiteMmaAccEmpty));
                 if (!ok) break;
-                if (lane == 0) ATTNW_STAMP(3 + q, it);
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>((q * 2 + buf) * kTile);
                 const uint32_t a_addr = q_addr + static_cast<uint32_t>(q * L::kTileBytes);
@@ -387,7 +366,6 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             if (!ok) break;
             if (ptx::elect_one()) ptx::umma_commit(&bars->k_empty[s]);  // the stage is free once these MMAs have read it
             __syncwarp();
-            if (lane == 0) ATTNW_STAMP(5, it);
         }
     } else if (warp < kSoftmaxWarps) {
         // ================= Softmax warps =================
@@ -404,18 +382,14 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             float mb = smax;         // the offset the exponentials in l are relative to: fl(smax * c2), finite from the start
             float l = 0.0f;          // running sum of 2^(c2 * s - mb) over this thread's columns
             bool ok = true;
-            const bool stamp = (warp & 7) == 0 && lane == 0;
-            (void)stamp;
 
             // ---- statistics pass (Eq. 1: m_i and the denominator), online over key tiles ----
             for (int it = 0; it < T; ++it) {
                 const int buf = it & 1;
-                if (stamp) ATTNW_STAMP(6 + q * 4, it);
                 ok = fused_wait(&bars->s_full[q][buf], static_cast<uint32_t>(it >> 1) & 1u, abort_flag,
                                 kSiteSoftmaxStats);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (stamp) ATTNW_STAMP(7 + q * 4, it);
                 ptx::tc_fence_after_sync();
 #pragma unroll 1
                 for (int c = 0; c < kHalf / kChunk; ++c) {
@@ -425,7 +399,6 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         ptx::tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(&bars->s_empty[q][buf]);
-                        if (stamp) ATTNW_STAMP(8 + q * 4, it);
                     }
                     const int valid = N - (kt0 + it) * kTile - half * kHalf - c * kChunk;  // columns of this chunk that exist
                     const bool ragged = valid < kChunk;
@@ -455,7 +428,6 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     l += ragged ? sum_exp2_chunk<kPolyStats, true>(s, c2c2, -mb, valid)
                                 : sum_exp2_chunk<kPolyStats, false>(s, c2c2, -mb, valid);
                 }
-                if (stamp) ATTNW_STAMP(9 + q * 4, it);
             }
 
             // ---- merge the two column halves of each row (both threads end with the same values) ----
@@ -512,12 +484,10 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
             for (int it = T; ok && it < total_iters; ++it) {
                 const int kt = kt0 + it - T;
                 const int buf = it & 1;
-                if (stamp) ATTNW_STAMP(6 + q * 4, it);
                 ok = fused_wait(&bars->s_full[q][buf], static_cast<uint32_t>(it >> 1) & 1u, abort_flag,
                                 kSiteSoftmaxNorm);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (stamp) ATTNW_STAMP(7 + q * 4, it);
                 ptx::tc_fence_after_sync();
                 // the previous store must have read the staging buffer before anyone overwrites it
                 if (issuer) {
@@ -539,7 +509,6 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                         ptx::tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(&bars->s_empty[q][buf]);
-                        if (stamp) ATTNW_STAMP(8 + q * 4, it);
                     }
 #pragma unroll
                     for (int j = 0; j < kChunk; j += 2) {
@@ -604,7 +573,6 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                     }
                     ++n_tiles;
                 }
-                if (stamp) ATTNW_STAMP(9 + q * 4, it);
             }
             if (lane == 0) ptx::bulk_wait_group<0>();
         }
@@ -621,18 +589,6 @@ attnw_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
-#ifdef ATTNW_CTA_CLOCK
-    if (threadIdx.x == 0 && blockIdx.x < 4096) {
-        long long ns1;
-        int sm;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns1));
-        asm volatile("mov.u32 %0, %%smid;" : "=r"(sm));
-        g_attnw_cta_clock[blockIdx.x][0] = clock64() - cc0;
-        g_attnw_cta_clock[blockIdx.x][1] = ns1 - ns0;
-        g_attnw_cta_clock[blockIdx.x][2] = sm;
-        g_attnw_cta_clock[blockIdx.x][3] = ns0;
-    }
-#endif
 }
 
 }  // namespace attnw

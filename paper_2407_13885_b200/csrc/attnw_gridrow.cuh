@@ -4,9 +4,14 @@
 // The paper lays the score matrix out over a grid of cores; the cores of one grid row hold the pieces of the
 // same rows of scores, compute LOCAL row maxima and sums and exchange them to obtain the GLOBAL ones before
 // normalising (Section VII; Eq. 1).  Here a group of C = ceil(N / 256) <= 16 CTAs owns a 128-row block of one
-// head.  CTA r of the group keeps the 128 x 256 slab of scores for keys [256 r, 256 r + 256) in HALF of its
-// tensor memory, so two row blocks are in flight per CTA: while the statistics of one cross the group, the
-// exponentials of the other keep the MUFU busy.  Tensor cores and exponentials run once per element.
+// head; CTA r of the group works on the 128 x 256 slab of scores for keys [256 r, 256 r + 256).  Tensor cores
+// and exponentials run once per element, and three row blocks are in flight per CTA:
+//   tensor-memory columns [0, 256)    two landing slots of 128 columns: the MMA writes float32 scores here; a slot
+//                                     goes back to the MMA issuer as soon as its scores are in registers
+//   tensor-memory columns [256, 512)  two packed regions (one per stream = row blocks of equal parity): the
+//                                     exponentials as f16 pairs, waiting for the row's statistics
+// so the next row block's scores are computed, and its exponentials taken, while the statistics of the previous
+// ones cross the group.  (f16 keeps 11 bits of e in [0, 1]: 5e-4 relative, next to the 2e-3 of the bf16 result.)
 //
 // Groups are not hardware clusters (clusters of 8 or 16 CTAs cannot occupy every SM): the grid is launched
 // cooperatively with one CTA per SM, consecutive CTAs form a group, and the 16-byte (offset, sum) pair of a row
@@ -14,19 +19,25 @@
 // pair once both tags name the row block it is waiting for.  No fence, no flag, no atomics: the tag arrives
 // with the value in one 8-byte store.  Every poll is bounded.
 //
-// Roles of a CTA (512 threads, 16 warps; warp w may touch TMEM lanes 32 (w % 4) ...):
-//   warps 0-3   exponentials of stream 0 (row blocks 0, 2, 4, ... of the group's list): a thread owns one row;
-//               per 128-column slot as its MMA completes, in chunks of 32 columns: running maximum,
-//               e = 2^(c s - mb) written back over s in TMEM, running sum; then the row's (mb, l) is posted
-//   warps 4-7   the same for stream 1 (row blocks 1, 3, 5, ...), on the other half of tensor memory
-//   warps 8-11  normalise: a thread owns one row; waits for the C pairs of the row, forms M and 1/L - every
-//               CTA reduces redundantly, as the paper's kernel does -, then p = e * 2^(mb_chunk - M) / L,
-//               rounded to bf16, staged in 128-row boxes; hands each slot back to the MMA issuer
-//   warp 12     TMA producer: the CTA's key slab once per head (it stays in shared memory while the group
-//               walks the head's row blocks), one 32 KB query tile per row block
-//   warp 13     tcgen05.mma issuer (one elected lane), 128 x 128 x 16 per instruction
-//   warp 14     store issuer: one TMA store per filled box; P is written exactly once
+// Roles of a CTA (640 threads, 20 warps; warp w may touch TMEM lanes 32 (w % 4) ...):
+//   warps 0-7    exponentials, all eight on ONE row block at a time: two threads per row, thread (row, p) takes the
+//                64-column boxes p and p + 2 of the slab: scores to registers, maximum, offset mb, e = 2^(c s - mb),
+//                sum, e packed to f16 pairs into the stream's packed region; the thread's (mb, l) to shared memory
+//   warps 8-11   normalise, stream 0 (12-15: stream 1): a thread owns one row; merges the row's two halves, posts
+//                the pair, waits for the C pairs of the row, forms M and 1/L - every CTA reduces redundantly, as
+//                the paper's kernel does -, then per box p = e * 2^(mb_box - M) / L (one mixed-precision FMA per
+//                element unpacks and scales), rounded to bf16, staged in 128-row boxes
+//   warp 16      TMA producer: the CTA's key slab once per head (it stays in shared memory while the group walks
+//                the head's row blocks), one 32 KB query tile per row block
+//   warp 17      tcgen05.mma issuer (one elected lane), 128 x 128 x 16 per instruction
+//   warps 18-19  store issuers, one per stream: one TMA store per filled box; P is written exactly once
 // Valid for N <= 4096 keys and bf16 output.
+//
+// With -DATTNW_TIMELINE=<CTA> one lane per role of that CTA stamps clock64() per row block (events, by index):
+//   13 MMA of the block issued | 0 exponentials begin, 2 slot 0 ready, 17/20 load of box k, 16/19 maximum known,
+//   18/21 exponentials of box k done, 24/26 packed e stored, 4 halves posted | 10 normalise begins to wait,
+//   6 halves seen + pair posted, 11 all pairs seen, 12 box 0 read, 14/15/8/9 box 2 read / staging free / staged /
+//   handed to the store issuer, 7 block done.
 #pragma once
 #include "attnw_resident.cuh"
 
@@ -40,12 +51,9 @@ constexpr int kPackedCol0 = kSlabCols;               // packed exponentials: col
 constexpr int kPackedCols = kSlabCols / 2;           // two f16 per 32-bit column
 constexpr int kBoxCols = 64;                         // columns of one staged store box (128 bytes of bf16)
 constexpr int kChunksPerBlock = kSlabCols / kChunk;  // 32-column chunks, each with its own offset
-#ifndef ATTNW_GR_THREADS
-#define ATTNW_GR_THREADS 640
-#endif
-constexpr int kThreads = ATTNW_GR_THREADS;           // 8 exponential + 8 normalise warps, producer, MMA issuer, store issuer
+constexpr int kThreads = 640;                        // 8 exponential + 8 normalise warps, producer, MMA issuer, 2 store issuers
 constexpr int kNormWarp0 = 8;
-constexpr int kNormGroups = 2;                         // normalise warpgroups: one per stream, or one for both
+constexpr int kNormGroups = 2;                       // normalise warpgroups: one per stream
 constexpr int kProducerWarpG = kNormWarp0 + 4 * kNormGroups;
 constexpr int kMmaWarpG = kProducerWarpG + 1;
 constexpr int kStoreWarpG = kProducerWarpG + 2;
@@ -98,22 +106,6 @@ struct Barriers {
     uint32_t prior_failure;
 };
 static_assert(sizeof(Barriers) <= 512, "barrier block must fit its slot");
-
-#ifdef ATTNW_TIMELINE
-__device__ unsigned long long g_attnw_gt[160][3][160];  // [CTA][posted / statistics seen / normalise begin][row block]: %globaltimer
-#define ATTNW_GT(ev, it)                                                                        \
-    do {                                                                                        \
-        if (blockIdx.x < 160 && (it) < 160) {                                                   \
-            unsigned long long t_;                                                              \
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                              \
-            g_attnw_gt[blockIdx.x][ev][it] = t_;                                                \
-        }                                                                                       \
-    } while (0)
-#else
-#define ATTNW_GT(ev, it) \
-    do {                 \
-    } while (0)
-#endif
 
 __device__ __forceinline__ void st_message(uint4* p, float a, float b, uint32_t tag) {
     asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(__float_as_uint(a)), "r"(tag),
@@ -192,13 +184,6 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
-#ifdef ATTNW_TIMELINE
-    if (threadIdx.x == 0 && blockIdx.x < 160) {
-        uint32_t smid;
-        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-        g_attnw_gt[blockIdx.x][2][159] = smid;
-    }
-#endif
     const bool run = bars->prior_failure == 0u && n_items > 0;  // an earlier launch step gave up: skip the work
 
     if (run && warp == kProducerWarpG) {
@@ -300,8 +285,7 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             const uint64_t stream_out = ptx::policy_evict_first();
             const uint32_t out_base = ptx::smem_u32(smem + L::kOutOff);
             bool ok = true;
-            constexpr int kStoreWarps = (kThreads >= 640) ? 2 : 1;  // one store issuer per stream, or one for both
-            for (int i = warp - kStoreWarpG; ok && i < n_items; i += kStoreWarps) {
+            for (int i = warp - kStoreWarpG; ok && i < n_items; i += 2) {  // one store issuer per stream
                 const int gi = begin + i, bh = gi / T, rb = gi % T;
                 const int s = i & 1;
                 const uint32_t ring = s ? L::kRing1 : L::kRing0, base = s ? L::kRing0 : 0;
@@ -322,10 +306,9 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             ptx::bulk_wait_group<0>();
         }
     } else if (run && warp < kNormWarp0) {
-        // ================= exponential warps: TMEM lane quarter = warp % 4, chunk parity = warp / 4 =================
+        // ================= exponential warps: TMEM lane quarter = warp % 4, box parity = warp / 4 =================
         // All eight warps work on ONE row block at a time (both streams in turn): two threads per row, one taking the
-        // even and one the odd 32-column chunks, so a row block's exponentials take half as long as with a warp per
-        // stream and the MUFU of every scheduler is fed by two warps in the same phase.
+        // even and one the odd 64-column boxes, so that every scheduler has two warps feeding its MUFU.
         const int par = warp >> 2;
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
@@ -339,9 +322,6 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const bool stamp = warp == 0 && lane == 0;
         (void)stamp;
         bool ok = true;
-#ifdef ATTNW_GR_STAGGER
-        if (par == 1) __nanosleep(ATTNW_GR_STAGGER);
-#endif
         for (int i = 0; ok && i < n_items; ++i) {
             const int s = i & 1;
             const uint32_t u = static_cast<uint32_t>(i) >> 1;
@@ -472,14 +452,12 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             if (!ok) break;
             ptx::tc_fence_after_sync();
             if (stamp) ATTNW_STAMP(6, i);
-            if (stamp) ATTNW_GT(2, i);
             // the two halves of the row are merged and the row's local pair goes to every CTA of the group (through L2)
             {
                 const float2 pa = part[(s * 2 + 0) * kTile + row], pb = part[(s * 2 + 1) * kTile + row];
                 const float mc = fmaxf(pa.x, pb.x);
                 const float lc = pa.y * ptx::ex2_approx(pa.x - mc) + pb.y * ptx::ex2_approx(pb.x - mc);
                 st_message(my_msg + (i & (kXchgDepth - 1)) * kTile, mc, lc, tag_base + static_cast<uint32_t>(i) + 1u);
-                if (stamp) ATTNW_GT(0, i);
             }
             // ---- global statistics of the row: wait for the C pairs, reduce them (redundantly in every CTA) ----
             // Entry reuse: row blocks i and i + 4 share entries.  A CTA posts block i + 4 after it has read the
@@ -492,33 +470,6 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 const uint4* src = group_msg + (i & (kXchgDepth - 1)) * kTile;
                 uint4 v[kMaxGroupCtas];
                 const long long t0 = clock64();
-                // Gate: while the group is still working, a lane watches ONE pair (its own row, CTA lane % C) - one
-                // load per lane and round instead of C, so that waiting costs the load/store path next to nothing.
-#ifdef ATTNW_GR_GATE
-                {
-                    const uint4* gate = src + static_cast<size_t>(lane % group_ctas) * kXchgDepth * kTile;
-                    for (uint32_t spin = 1;; ++spin) {
-                        const uint4 g = ld_message(gate);
-                        if (__all_sync(0xffffffffu, g.y == tag && g.w == tag)) break;
-#ifndef ATTNW_GR_NOSLEEP
-                        __nanosleep(64);
-#endif
-                        if ((spin & 15u) == 0) {
-                            bool give_up = *abort_flag != 0u;
-                            if (!give_up && clock64() - t0 > kWaitLimitCycles) {
-                                *abort_flag = 1;
-                                atomicCAS(&g_attnw_status, 0u, 0x80000000u | kSiteGrExchange);
-                                give_up = true;
-                            }
-                            if (__any_sync(0xffffffffu, give_up)) {
-                                ok = false;
-                                break;
-                            }
-                        }
-                    }
-                    if (!ok) break;
-                }
-#endif
                 for (uint32_t spin = 1;; ++spin) {
                     // all loads first (entries beyond the group repeat its last CTA), then the tags
 #pragma unroll
@@ -543,7 +494,6 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 }
                 if (!ok) break;
                 if (stamp) ATTNW_STAMP(11, i);
-                if (stamp) ATTNW_GT(1, i);
                 m_row = __uint_as_float(v[0].x);
 #pragma unroll
                 for (int c = 1; c < kMaxGroupCtas; ++c) m_row = fmaxf(m_row, __uint_as_float(v[c].x));
@@ -589,12 +539,7 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
                             for (int x = 0; x < 4; ++x) {
                                 float lo, hi;
-#ifdef ATTNW_GR_CVT_UNPACK
-                                ptx::unpack_f16x2(e[gg * 4 + x], lo, hi);
-                                ptx::unpack2(ptx::mul2(ptx::pack2(lo, hi), ptx::pack2(f[b], f[b])), lo, hi);
-#else
                                 ptx::scale_f16x2(e[gg * 4 + x], fh, lo, hi);
-#endif
                                 w[x] = ptx::pack_bf16x2(lo, hi);
                             }
                             ptx::st_shared_v4(my_row + ((static_cast<uint32_t>(gg) ^ sw) << 4), w[0], w[1], w[2], w[3]);

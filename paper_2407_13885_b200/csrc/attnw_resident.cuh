@@ -128,7 +128,7 @@ __device__ __forceinline__ float exp2_chunk_inplace(float (&s)[kChunk], uint64_t
 // clusters work on neighbouring row blocks of one head, so its keys stay hot in L2).  Every role of every CTA
 // of the cluster walks the same list.
 // OWNER = false: every CTA receives every CTA's pairs and reduces them itself (redundantly, as the paper's kernel
-// does).  OWNER = true: the alternative the paper names as future work (Section IX): the rows are dealt out to the
+// does).  OWNER = true: the alternative the paper names as future work (Section VIII): the rows are dealt out to the
 // CTAs (row i belongs to CTA i mod C); the owner receives the C pairs of its rows, reduces them once and sends
 // (M, 1/L) to every CTA - two hops of latency instead of one, C times fewer messages and reductions.
 template <int D, int CMAX, bool OWNER>
@@ -283,17 +283,11 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             const uint32_t out_base = ptx::smem_u32(smem + L::kOutOff);
             uint32_t n = 0;
             bool ok = true;
-#ifdef ATTNW_TIMELINE
-            long long acc_filled = 0, acc_read = 0, tq;
-#endif
             for (int g = cluster; ok && g < total_items; g += n_clusters) {
                 const int bh = g / T, rb = g % T;
                 for (int t = 0; ok && t < n_sub; ++t)
                     for (int h = 0; h < 2; ++h, ++n) {
                         const uint32_t box = n % kStageBoxes, use = n / kStageBoxes;
-#ifdef ATTNW_TIMELINE
-                        tq = clock64();
-#endif
                         if (!fused_wait(&bars->out_filled[box], use & 1u, abort_flag, kSiteResStageFilled)) {
                             ok = false;
                             break;
@@ -304,28 +298,14 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                         if (out_col < N)
                             ptx::tma_store_3d(&tm_p, out_base + box * kBoxBytes, out_col, rb * kTile, bh, stream_out);
                         ptx::bulk_commit_group();
-#ifdef ATTNW_TIMELINE
-                        acc_filled += clock64() - tq;
-                        tq = clock64();
-#endif
                         // Once at most kStoreLag stores are still reading, store n - kStoreLag has read its ring entry:
                         // that entry is free for its next use, kStageBoxes - kStoreLag boxes ahead of the Softmax
                         // warps.  (An entry's first use needs no arrival: it starts free, and the Softmax warps
                         // wait for phase use - 1 of out_free before use >= 1.)
                         ptx::bulk_wait_group_read<kStoreLag>();
                         if (n >= kStoreLag) ptx::mbar_arrive(&bars->out_free[(n - kStoreLag) % kStageBoxes]);
-#ifdef ATTNW_TIMELINE
-                        acc_read += clock64() - tq;
-#endif
                     }
             }
-#ifdef ATTNW_TIMELINE
-            if (blockIdx.x == ATTNW_TIMELINE) {
-                g_attnw_timeline[6][0] = acc_filled;
-                g_attnw_timeline[6][1] = acc_read;
-                g_attnw_timeline[6][2] = n;
-            }
-#endif
             ptx::bulk_wait_group<0>();
         }
     } else if (run && warp < kSoftmaxWarps) {
@@ -347,8 +327,6 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         float2* stat = reinterpret_cast<float2*>(smem + L::kStatOff);
         const uint32_t out_base = ptx::smem_u32(smem + L::kOutOff);
         const uint32_t sw = static_cast<uint32_t>(row & 7);
-        const bool stamp = warp == 0 && lane == 0;
-        (void)stamp;
         bool ok = true;
 
         // sweep-1 state of the row block being accumulated
@@ -360,7 +338,6 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             ok = __all_sync(0xffffffffu, fused_wait(&bars->s_full[t], item & 1u, abort_flag, kSiteResSFull));
             if (!ok) return;
             ptx::tc_fence_after_sync();
-            if (stamp) ATTNW_STAMP(8 + t, item);
             float s[kChunk];
             load_chunk(t_base + static_cast<uint32_t>(t * kTile), s);
             const int valid = width - t * kTile - cq * kChunk;  // columns of this chunk that exist (may be <= 0)
@@ -399,7 +376,6 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         auto post_partials = [&](uint32_t item) {
             ptx::tmem_wait_st();
             if (!ok) return;
-            if (stamp) ATTNW_STAMP(1, item);
             const uint32_t par = item & 1u;
             part[cq * kTile + row] = make_float2(mb, l);
             __syncwarp();
@@ -461,7 +437,6 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                     }
                 }
             }
-            if (stamp) ATTNW_STAMP(3, item);
         };
 
         // walk the list of row blocks with one block of look-ahead
@@ -491,7 +466,6 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             if (cq == 0) {
                 ok = __all_sync(0xffffffffu, fused_wait(&bars->x_full[par], (item_n >> 1) & 1u, abort_flag, kSiteResExchange));
                 if (!ok) break;
-                if (stamp) ATTNW_STAMP(4, item_n);
                 if constexpr (!OWNER) {
                     // all exchange slots are read at once (independent loads); slots beyond the cluster are ignored
                     float2 pc[CMAX];
@@ -532,13 +506,11 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             for (int t = 0; t < kSlots; ++t) {
                 if (t < n_sub && ok) {
                     // ---- sweep 2 of slot t: normalise, round, stage, store; hand the slot back ----
-                    if (stamp && t == 1) ATTNW_STAMP(0, item_n);
                     float e[kChunk];
                     load_chunk(t_base + static_cast<uint32_t>(t * kTile), e);
                     ptx::tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(&bars->slot_free[t]);
-                    if (stamp && t == 1) ATTNW_STAMP(2, item_n);
                     // staging box of this (row block, slot, column half): ring entry box_n % kStageBoxes; the store
                     // that last used the entry must have read it before anyone overwrites it
                     const uint32_t n_box = box_n * 2u + static_cast<uint32_t>(h);  // boxes alternate between the halves
@@ -546,7 +518,6 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                     const uint32_t my_row = out_base + box * kBoxBytes + static_cast<uint32_t>(row * 128);
                     ok = __all_sync(0xffffffffu, fused_wait(&bars->out_free[box], (use & 1u) ^ 1u, abort_flag,
                                                             kSiteResStageFree));
-                    if (stamp && t == 1) ATTNW_STAMP(5, item_n);
                     if (ok) {
                         const uint64_t ff = ptx::pack2(f_slot[t], f_slot[t]);
 #pragma unroll
@@ -564,7 +535,6 @@ attnw_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
                         if (lane == 0) ptx::mbar_arrive(&bars->out_filled[box]);
                         ++box_n;
                     }
-                    if (stamp) ATTNW_STAMP(12 + t, item_n);
                 }
                 // ---- sweep 1 of slot t - kS1Lag of the next row block: its MMA started when that slot was freed,
                 //      kS1Lag slots of sweep 2 ago, and has had time to finish ----

@@ -1,6 +1,6 @@
 // Queries and keys from the inputs for sm_100a: Q_h = X W^Q_h, K_h = X W^K_h for every head in one launch - the
 // linear transformation in front of the attention weights (Section IV), which the paper leaves to the vendor's
-// matmul and names as a step to bring into its own code (Section IX).  The output is written head-major
+// matmul and names as a step to bring into its own code (Section VIII).  The output is written head-major
 // ([B, H, N, d], bf16), exactly what attnw_fused and attn_fused read, so no transposition pass is needed.
 //
 // A plain dense contraction, so it runs on the tensor cores: a CTA owns a 256 x 256 tile of one of the two
