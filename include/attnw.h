@@ -60,6 +60,29 @@ int attnw_fused(const void* Q, const void* K, void* P, int B, int H, int N, int 
 int attnw_fused_f32(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream);
 
 /*
+ * attnw_fused_noalloc: attnw_fused (bfloat16 P) for callers that cannot allocate device memory.  The paper has no
+ * counterpart; this is a property of the library, not of the method.
+ *
+ * Who needs it: code that runs where cudaMalloc is not allowed or not wanted - inside a framework whose memory pool
+ * owns all device memory, in a real-time loop that must not take the allocator's lock or its implicit
+ * synchronisation, or in a process that has handed the rest of the GPU's memory to someone else.  attnw_fused itself
+ * allocates its exchange area with cudaMalloc the first time it runs the grid-row kernel on a device; this entry
+ * point never calls cudaMalloc, cudaFree or any other allocating routine.  Its exchange area is a fixed array inside
+ * the library's device image (1.25 MiB, present on every GPU that loads the library until the process exits).
+ *
+ * Arguments, layout and result are those of attnw_fused.  Limits, each refused with a status code and no launch:
+ *   N <= 4096 (ATTNW_ERR_UNSUPPORTED beyond: one group of the grid-row kernel holds at most 4096 keys), and a device
+ *   on which one group fits among at most 160 resident CTAs (the array has entries for 160; a B200 uses 144 or 148).
+ * First call on a device: looks up the array's device address (cudaGetSymbolAddress) and the device's properties.
+ *   Make that first call before any stream capture begins.
+ * Every call on a device shares the one array, which keeps what the previous call left in it; the messages carry
+ *   tags that no later call repeats, so nothing has to be cleared between calls (after about 4e9 row blocks the tags
+ *   start over and the call first clears the array, in stream order).  Two calls that overlap in time on one device
+ *   - different streams with nothing ordering them - race on the array: order them, or use attnw_fused for one.
+ */
+int attnw_fused_noalloc(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream);
+
+/*
  * attn_fused: O[b,h,i,c] = sum_j P[b,h,i,j] * V[b,h,j,c] with P as defined for attnw_fused - Attention(Q, K, V) of
  * Section IV, the product with V that Section VIII leaves as future work - in one kernel; neither the scores nor the
  * weights reach HBM.

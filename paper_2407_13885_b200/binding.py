@@ -26,6 +26,7 @@ SIGNATURES = {
     "attnw_fused_host": (_int, [_vp, _vp, _vp, _int, _int, _int, _int, _float, _int]),
     "softmax_rows_host": (_int, [_vp, _vp, _ll, _ll, _int]),
     "attnw_host_release": (_int, []),
+    "attnw_fused_noalloc": (_int, [_vp, _vp, _vp, _int, _int, _int, _int, ctypes.c_float, _vp]),
     "attnw_query_status": (_int, [_vp, ctypes.POINTER(ctypes.c_uint)]),
     "attnw_selftest_wait_timeout": (_int, [_ll, _vp]),
     "attnw_set_fused_variant": (_int, [_int]),
@@ -262,3 +263,25 @@ def selftest_wait_timeout(limit_cycles: int = 1_000_000, stream=None) -> None:
     """Launches the failure-path self-test: one warp waits ``limit_cycles`` SM clocks on a barrier nobody arrives on,
     gives up and records site 127 in the device status word (see ``attnw_selftest_wait_timeout``)."""
     _check(lib.attnw_selftest_wait_timeout(int(limit_cycles), _stream_ptr(stream)), "attnw_selftest_wait_timeout")
+
+
+def attnw_fused_noalloc(Q: torch.Tensor, K: torch.Tensor, scale: float, P: torch.Tensor | None = None,
+                        stream=None) -> torch.Tensor:
+    """``attnw_fused`` (bfloat16 P, N <= 4096) through the entry point that never allocates device memory: for callers
+    that may not call cudaMalloc (a memory pool owns the device, or the call sits in a latency-critical loop).  The
+    output tensor is still the caller's (or allocated here by torch, outside the library)."""
+    _require_cuda(Q, "Q", torch.bfloat16)
+    _require_cuda(K, "K", torch.bfloat16)
+    if Q.dim() != 4 or Q.shape != K.shape:
+        raise ValueError("Q and K must both be [B, H, N, d]")
+    B, H, N, d = Q.shape
+    if P is None:
+        P = torch.empty((B, H, N, N), dtype=torch.bfloat16, device=Q.device)
+    else:
+        _require_cuda(P, "P", torch.bfloat16)
+        if tuple(P.shape) != (B, H, N, N):
+            raise ValueError("P must be [B, H, N, N] in bfloat16")
+    with torch.cuda.device(Q.device):
+        _check(lib.attnw_fused_noalloc(Q.data_ptr(), K.data_ptr(), P.data_ptr(), B, H, N, d, float(scale),
+                                       _stream_ptr(stream)), "attnw_fused_noalloc")
+    return P

@@ -732,6 +732,109 @@ int staging_reserve(HostStaging* st, int slot, int which, size_t bytes) {
 
 constexpr unsigned long long kHostChunkBytes = 256ull << 20;  // target size of one staged piece of P
 
+// ---- attnw_fused_noalloc: the grid-row kernel with its exchange area in a static device array ----------------
+// Scratch of the entry point that allocates nothing: the exchange area of the grid-row kernel for a grid of up to
+// kNoAllocMaxCtas CTAs (messages of 16 bytes: [CTA][4 row blocks in flight][128 rows]) = 1.25 MiB, held by every
+// GPU that loads the library until the process exits.  In host code this name is only a stand-in for the symbol:
+// the device address comes from cudaGetSymbolAddress (noalloc_setup below) and is what the kernel is given.
+constexpr int kNoAllocMaxCtas = 160;
+static __device__ __align__(256) uint4 g_noalloc_xchg[kNoAllocMaxCtas * gr::kXchgDepth * kTile];
+
+struct NoAllocState {
+    bool ready = false;
+    uint4* xchg = nullptr;   // device address of g_noalloc_xchg on this device
+    int sm_count = 0;
+    uint32_t tag = 0;        // next unused message tag of this device's array
+};
+NoAllocState g_noalloc[kMaxDevices];
+
+// Once per device, with that device current.  Returns an attnw_status.
+int noalloc_setup(NoAllocState** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(g_mutex);
+    NoAllocState& st = g_noalloc[dev];
+    if (!st.ready) {
+        int major = 0;
+        void* ptr = nullptr;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return ATTNW_ERR_CUDA;
+        }
+        if (major != 10) return ATTNW_ERR_UNSUPPORTED;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_xchg) != cudaSuccess || ptr == nullptr) {
+            (void)cudaGetLastError();
+            return ATTNW_ERR_CUDA;
+        }
+        st.xchg = static_cast<uint4*>(ptr);
+        st.tag = 0;  // the array is zero when the module is loaded, and zero is never a tag
+        st.ready = true;
+    }
+    *out = &st;
+    return ATTNW_OK;
+}
+
+template <int D>
+int launch_gridrow_noalloc(NoAllocState* st, const void* Q, const void* K, void* P, int BH, int N, float scale,
+                           cudaStream_t stream) {
+    using L = gr::Smem<D>;
+    auto kernel = gr::attnw_gridrow_kernel<D>;
+    CUtensorMap tm_q, tm_k, tm_p;
+    int rc = encode_3d(&tm_q, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Q, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, K, D, N, BH, 64, kTile);
+    if (rc == ATTNW_OK) rc = encode_3d(&tm_p, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, P, N, N, BH, 64, kTile);
+    if (rc != ATTNW_OK) return rc;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamicBytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    const int group_ctas = (N + gr::kSlabCols - 1) / gr::kSlabCols;
+    const long long total_items = static_cast<long long>(BH) * ((N + kTile - 1) / kTile);
+    if (total_items > INT_MAX) return ATTNW_ERR_BAD_SHAPE;
+    // one CTA per SM, whole groups only, and never more CTAs than the static array has entries for
+    const int max_ctas = st->sm_count < kNoAllocMaxCtas ? st->sm_count : kNoAllocMaxCtas;
+    if (max_ctas < group_ctas) return ATTNW_ERR_UNSUPPORTED;
+    int n_groups = max_ctas / group_ctas;
+    if (n_groups > total_items) n_groups = static_cast<int>(total_items);
+    uint32_t tag_base = 0;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        const uint32_t longest = static_cast<uint32_t>((total_items + n_groups - 1) / n_groups);
+        if (st->tag > 0xffffffffu - longest - 1u) {
+            // the tags are used up (after about 4e9 row blocks): start again from a cleared array, in stream order
+            if (cudaMemsetAsync(st->xchg, 0, sizeof(g_noalloc_xchg), stream) != cudaSuccess) {
+                (void)cudaGetLastError();
+                return ATTNW_ERR_CUDA;
+            }
+            st->tag = 0;
+        }
+        tag_base = st->tag;
+        st->tag += longest;
+    }
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(gr::kThreads, 1, 1);
+    cfg.gridDim = dim3(static_cast<unsigned>(n_groups * group_ctas), 1, 1);
+    cfg.dynamicSmemBytes = L::kDynamicBytes;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const float scale_log2e = static_cast<float>(static_cast<double>(scale) * 1.4426950408889634074);
+    if (cudaLaunchKernelEx(&cfg, kernel, tm_q, tm_k, tm_p, N, static_cast<int>(total_items), group_ctas, n_groups, scale_log2e,
+                           st->xchg, tag_base) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ATTNW_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ATTNW_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -778,6 +881,20 @@ int attnw_set_attn_variant(int variant) {
 
 int attnw_fused(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream) {
     return fused_entry<__nv_bfloat16>(Q, K, P, B, H, N, d, scale, stream);
+}
+
+int attnw_fused_noalloc(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream) {
+    int rc = validate_fused(Q, K, P, B, H, N, d, scale, 2);
+    if (rc != ATTNW_OK) return rc;
+    if (N > gr::kMaxN) return ATTNW_ERR_UNSUPPORTED;  // beyond what the static exchange area and one group can serve
+    NoAllocState* st = nullptr;
+    rc = noalloc_setup(&st);
+    if (rc != ATTNW_OK) return rc;
+    rc = load_encoder();
+    if (rc != ATTNW_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    return d == 64 ? launch_gridrow_noalloc<64>(st, Q, K, P, B * H, N, scale, s)
+                   : launch_gridrow_noalloc<128>(st, Q, K, P, B * H, N, scale, s);
 }
 
 int attnw_fused_f32(const void* Q, const void* K, void* P, int B, int H, int N, int d, float scale, void* stream) {
