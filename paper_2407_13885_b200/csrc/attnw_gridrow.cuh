@@ -22,9 +22,9 @@
 // Roles of a CTA (640 threads, 20 warps; warp w may touch TMEM lanes 32 (w % 4) ...):
 //   warps 0-7    exponentials, all eight on ONE row block at a time: two threads per row, thread (row, p) takes the
 //                64-column boxes p and p + 2 of the slab: scores to registers, maximum, offset mb, e = 2^(c s - mb),
-//                sum, e packed to f16 pairs into the stream's packed region; the thread's (mb, l) to shared memory
-//   warps 8-11   normalise, stream 0 (12-15: stream 1): a thread owns one row; merges the row's two halves, posts
-//                the pair, waits for the C pairs of the row, forms M and 1/L - every CTA reduces redundantly, as
+//                sum, e packed to f16 pairs into the stream's packed region; the thread's (mb, l) to shared memory;
+//                the second of a row's two warps to finish merges the halves and posts the row's pair
+//   warps 8-11   normalise, stream 0 (12-15: stream 1): a thread owns one row; waits for the C pairs of the row, forms M and 1/L - every CTA reduces redundantly, as
 //                the paper's kernel does -, then per box p = e * 2^(mb_box - M) / L (one mixed-precision FMA per
 //                element unpacks and scales), rounded to bf16, staged in 128-row boxes
 //   warp 16      TMA producer: the CTA's key slab once per head (it stays in shared memory while the group walks
@@ -101,6 +101,7 @@ struct Barriers {
     uint64_t pk_free[2][kSlabCols / kBoxCols];              // [stream][box]: the packed exponentials have been read
     uint64_t posted[2];
     uint64_t out_free[6], out_filled[6];
+    uint32_t halves_done[2][4];  // [stream][TMEM lane quarter]: exponential warps that have finished a row's halves (never reset)
     uint32_t tmem_base;
     uint32_t abort_flag;
     uint32_t prior_failure;
@@ -167,6 +168,7 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             ptx::mbar_init(&bars->out_free[b], 1);
             ptx::mbar_init(&bars->out_filled[b], 4);
         }
+        for (int x = 0; x < 8; ++x) (&bars->halves_done[0][0])[x] = 0;
         bars->abort_flag = 0;
         bars->prior_failure = *reinterpret_cast<volatile unsigned int*>(&g_attnw_status);
         ptx::mbar_fence_init();
@@ -319,6 +321,7 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const uint64_t c2c2 = ptx::pack2(c2, c2);
         float* mbc_all = reinterpret_cast<float*>(smem + L::kMbcOff);
         float2* part_all = reinterpret_cast<float2*>(smem + L::kPartOff);
+        uint4* my_msg = xchg + (static_cast<size_t>(blockIdx.x) * kXchgDepth) * kTile + row;
         const bool stamp = warp == 0 && lane == 0;
         (void)stamp;
         bool ok = true;
@@ -420,6 +423,22 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             }
             if (!ok) break;
             part_all[(s * 2 + par) * kTile + row] = make_float2(mb, l);  // this thread's half of the row
+            // The second of the two warps to get here merges the halves and posts the row's pair to every CTA of the
+            // group (through L2) at once: the exchange must not wait for a normalise warp to become free.
+            __threadfence_block();
+            __syncwarp();
+            uint32_t before = 0;
+            if (lane == 0) before = atomicAdd(&bars->halves_done[s][quarter], 1u);
+            before = __shfl_sync(0xffffffffu, before, 0);
+            if (before & 1u) {
+                __threadfence_block();
+                const volatile float* pv = reinterpret_cast<const volatile float*>(part_all);
+                const float pax = pv[2 * ((s * 2 + 0) * kTile + row)], pay = pv[2 * ((s * 2 + 0) * kTile + row) + 1];
+                const float pbx = pv[2 * ((s * 2 + 1) * kTile + row)], pby = pv[2 * ((s * 2 + 1) * kTile + row) + 1];
+                const float mc = fmaxf(pax, pbx);
+                const float lc = pay * ptx::ex2_approx(pax - mc) + pby * ptx::ex2_approx(pbx - mc);
+                st_message(my_msg + (i & (kXchgDepth - 1)) * kTile, mc, lc, tag_base + static_cast<uint32_t>(i) + 1u);
+            }
             ptx::tmem_wait_st();
             ptx::tc_fence_before_sync();
             __syncwarp();
@@ -436,8 +455,6 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const uint32_t sw = static_cast<uint32_t>(row & 7);
         const uint4* group_msg = xchg + (static_cast<size_t>(group) * group_ctas * kXchgDepth) * kTile + row;
         const float* mbc_all = reinterpret_cast<const float*>(smem + L::kMbcOff);
-        const float2* part = reinterpret_cast<const float2*>(smem + L::kPartOff);
-        uint4* my_msg = xchg + (static_cast<size_t>(blockIdx.x) * kXchgDepth) * kTile + row;
         const int last_cta = group_ctas - 1;
         const bool stamp = quarter == 0 && lane == 0;
         (void)stamp;
@@ -452,13 +469,6 @@ attnw_gridrow_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             if (!ok) break;
             ptx::tc_fence_after_sync();
             if (stamp) ATTNW_STAMP(6, i);
-            // the two halves of the row are merged and the row's local pair goes to every CTA of the group (through L2)
-            {
-                const float2 pa = part[(s * 2 + 0) * kTile + row], pb = part[(s * 2 + 1) * kTile + row];
-                const float mc = fmaxf(pa.x, pb.x);
-                const float lc = pa.y * ptx::ex2_approx(pa.x - mc) + pb.y * ptx::ex2_approx(pb.x - mc);
-                st_message(my_msg + (i & (kXchgDepth - 1)) * kTile, mc, lc, tag_base + static_cast<uint32_t>(i) + 1u);
-            }
             // ---- global statistics of the row: wait for the C pairs, reduce them (redundantly in every CTA) ----
             // Entry reuse: row blocks i and i + 4 share entries.  A CTA posts block i + 4 after it has read the
             // statistics of block i + 2, i.e. after EVERY CTA has posted block i + 2; a CTA's scores of block i + 2
