@@ -77,8 +77,8 @@ def run(cta: int = 1, heads: int = 64, n: int = 4096, d: int = 128, launches: in
             "mma_issue_to_exponentials_begin": span(13, 0),
         },
         "normalise_role": {
-            "halves_posted_to_seen": float(np.mean(buf[6, it] - buf[4, it])),
-            "post_and_wait_for_group": span(6, 11), "reduce_and_read_box0": span(11, 12),
+            "first_warp_done_to_block_visible_to_normalise": float(np.mean(buf[6, it] - buf[4, it])),
+            "wait_for_group": span(6, 11), "reduce_and_read_box0": span(11, 12),
             "box2_wait_staging": span(14, 15), "box2_scale_round_stage": span(15, 8), "box2_fence_and_hand_over": span(8, 9),
             "all_pairs_seen_to_block_done": span(11, 7),
         },
