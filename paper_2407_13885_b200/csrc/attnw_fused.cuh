@@ -121,9 +121,6 @@ __device__ __noinline__ bool fused_wait_slow(uint64_t* bar, uint32_t parity, vol
     const long long t0 = clock64();
     for (uint32_t spin = 1;; ++spin) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
-#ifdef ATTNW_WAIT_SLEEP
-        __nanosleep(ATTNW_WAIT_SLEEP);
-#endif
         if ((spin & 63u) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitLimitCycles) {
