@@ -142,10 +142,10 @@ int attnw_set_attn_variant(int variant);
  *   4  grid-row kernel: the SRAM-resident design on a cooperative grid of one CTA per SM.  Consecutive ceil(N/256)
  *      CTAs form a group (the cores of one grid row in Section VII) that owns a 128-row block; every CTA keeps its
  *      128 x 256 slab of scores in half of its tensor memory, so two row blocks are in flight per CTA, and the local
- *      row maxima and sums cross the group through L2 as tagged 16-byte messages in a per-device exchange area that
- *      the library allocates on first use (cudaMalloc; never inside a stream capture).  Serves bfloat16 P and
- *      N <= 4096; any other call then returns ATTNW_ERR_UNSUPPORTED.  Two such launches must not run on one device
- *      at the same time (they share the exchange area); launches on one stream, or ordered by events, are fine.
+ *      row maxima and sums cross the group through L2 as tagged 16-byte messages in per-device exchange areas (4.7 MB)
+ *      that the library allocates on first use (cudaMalloc; never inside a stream capture).  Serves bfloat16 P and
+ *      N <= 4096; any other call then returns ATTNW_ERR_UNSUPPORTED.  Launches take the exchange areas in turn, so calls on
+ *      different streams of one device are safe as long as fewer than four of them are in flight at once.
  * Returns ATTNW_ERR_BAD_SHAPE for any other value.
  */
 int attnw_set_fused_variant(int variant);

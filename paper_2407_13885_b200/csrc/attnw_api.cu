@@ -26,6 +26,9 @@ namespace {
 using namespace attnw;
 
 constexpr int kMaxDevices = 64;
+// Consecutive launches of the grid-row kernel use different exchange areas in turn: the last CTAs of one launch may still
+// be reading the pairs of their last row block when the next launch (which starts as soon as its whole grid fits) posts.
+constexpr int kGridrowAreas = 4;
 constexpr uint32_t kSiteSelfTest = 127;  // wait site of attnw_selftest_wait_timeout (low byte of the status word)
 
 // Not part of any product path: one thread waits, with the caller's limit, on an mbarrier that nobody arrives on,
@@ -81,6 +84,7 @@ struct DeviceInfo {
     uint4* gridrow_xchg = nullptr;
     int gridrow_xchg_ctas = 0;
     uint32_t gridrow_tag = 0;
+    unsigned gridrow_launches = 0;  // selects one of kGridrowAreas exchange areas in turn
 };
 std::mutex g_split_mutex;
 DeviceInfo g_devices[kMaxDevices];
@@ -384,7 +388,7 @@ int launch_gridrow(DeviceInfo* dev, const void* Q, const void* K, void* P, int B
             // first use on this device: the exchange area, zero so that no entry carries a valid tag
             if (dev->gridrow_xchg) cudaFree(dev->gridrow_xchg);
             dev->gridrow_xchg = nullptr;
-            const size_t bytes = static_cast<size_t>(max_ctas) * gr::kXchgDepth * kTile * sizeof(uint4);
+            const size_t bytes = static_cast<size_t>(kGridrowAreas) * max_ctas * gr::kXchgDepth * kTile * sizeof(uint4);
             void* p = nullptr;
             if (cudaMalloc(&p, bytes) != cudaSuccess || cudaMemset(p, 0, bytes) != cudaSuccess ||
                 cudaDeviceSynchronize() != cudaSuccess) {
@@ -396,7 +400,8 @@ int launch_gridrow(DeviceInfo* dev, const void* Q, const void* K, void* P, int B
             dev->gridrow_xchg_ctas = max_ctas;
             dev->gridrow_tag = 0;
         }
-        xchg = dev->gridrow_xchg;
+        xchg = dev->gridrow_xchg + static_cast<size_t>(dev->gridrow_launches++ % kGridrowAreas) * dev->gridrow_xchg_ctas *
+                                       gr::kXchgDepth * kTile;
         // tags tag_base + 1 ... tag_base + (longest list) belong to this launch; 0 is never a tag
         const uint32_t longest = static_cast<uint32_t>((total_items + n_groups - 1) / n_groups);
         if (dev->gridrow_tag > 0xffffffffu - longest - 1u) dev->gridrow_tag = 0;
@@ -414,10 +419,12 @@ int launch_gridrow(DeviceInfo* dev, const void* Q, const void* K, void* P, int B
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const float scale_log2e = static_cast<float>(static_cast<double>(scale) * 1.4426950408889634074);
-    if (cudaLaunchKernelEx(&cfg, kernel, tm_q, tm_k, tm_p, N, static_cast<int>(total_items), group_ctas, n_groups, scale_log2e,
-                           xchg, tag_base) != cudaSuccess) {
+    const cudaError_t launched = cudaLaunchKernelEx(&cfg, kernel, tm_q, tm_k, tm_p, N, static_cast<int>(total_items), group_ctas,
+                                                    n_groups, scale_log2e, xchg, tag_base);
+    if (launched != cudaSuccess) {
         (void)cudaGetLastError();
-        return ATTNW_ERR_CUDA;
+        // the grid does not fit at once after all (SMs taken away from this context): let the caller choose another kernel
+        return launched == cudaErrorCooperativeLaunchTooLarge ? ATTNW_ERR_UNSUPPORTED : ATTNW_ERR_CUDA;
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return ATTNW_OK;
