@@ -85,6 +85,7 @@ struct DeviceInfo {
     int gridrow_xchg_ctas = 0;
     uint32_t gridrow_tag = 0;
     unsigned gridrow_launches = 0;  // selects one of kGridrowAreas exchange areas in turn
+    int rc_clusters[2][17] = {};  // resident clusters of 1..16 CTAs of the register-cluster row kernel, [P is float32][CTAs]
 };
 std::mutex g_split_mutex;
 DeviceInfo g_devices[kMaxDevices];
@@ -678,11 +679,11 @@ int rows_entry(const void* S, void* P, long long rows, long long cols, void* str
     if (variant == 1 && cols > srs::kMaxCols) return ATTNW_ERR_UNSUPPORTED;
     // Longer rows can be kept in the shared memory of a CTA or of a cluster (caching form).  By default that is done
     // where it is the faster way (measured): from 8192 columns on - there the register tier needs a whole CTA of 1024
-    // threads per row and stops overlapping rows - with one CTA or a cluster of two; with larger clusters the cluster
-    // barrier of every row costs more than the second read of the two-read kernel.
+    // threads per row and stops overlapping rows - with one CTA, or a cluster of two up to 32768 columns; beyond, the
+    // cluster barrier of every row costs more than the second read (from L2) of the two-read kernel.
     const int smem_ctas = cols > kSoftmaxRowsSmemTierMinCols ? srs::cluster_ctas_for(cols) : 0;
-    const bool smem_default = smem_ctas == 1 || smem_ctas == 2;
-    if ((variant <= 1 && smem_default) || (variant == 1 && smem_ctas > 2)) {
+    const bool smem_default = smem_ctas == 1 || (smem_ctas == 2 && cols <= kSoftmaxRowsRegTierMaxCols);
+    if ((variant == 0 && smem_default) || (variant == 1 && smem_ctas >= 1)) {
         if (srs::launch<OutT>(static_cast<const float*>(S), static_cast<OutT*>(P), rows, cols, dev->sm_count,
                               static_cast<cudaStream_t>(stream)) == cudaSuccess) {
             g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -690,6 +691,18 @@ int rows_entry(const void* S, void* P, long long rows, long long cols, void* str
         }
         (void)cudaGetLastError();  // no cluster of that size on this device: fall through to the two-read kernel
         if (variant == 1) return ATTNW_ERR_UNSUPPORTED;
+    }
+    // Rows of 32769 to 262144 columns: kept in the registers of a cluster, one read and one write per element.
+    if (variant == 0 && cols > kSoftmaxRowsRegTierMaxCols && cols <= srs::kRcMaxCols) {
+        const int C = srs::rc_cluster_ctas_for(cols);
+        const cudaError_t ce = srs::launch_regcluster<OutT>(static_cast<const float*>(S), static_cast<OutT*>(P), rows, cols,
+                                                            &dev->rc_clusters[sizeof(OutT) == 4][C],
+                                                            static_cast<cudaStream_t>(stream));
+        if (ce == cudaSuccess) {
+            g_launches.fetch_add(1, std::memory_order_relaxed);
+            return ATTNW_OK;
+        }
+        (void)cudaGetLastError();  // no cluster of that size on this device: the two-read kernel
     }
     cudaError_t e = softmax_rows_launch<OutT>(static_cast<const float*>(S), static_cast<OutT*>(P), rows, cols,
                                               dev->sm_count, static_cast<cudaStream_t>(stream), variant == 3 ? 1 : (variant == 2 ? 2 : 0));

@@ -207,5 +207,195 @@ inline cudaError_t launch(const float* S, OutT* P, long long rows, long long col
     return launch_nt<OutT, 512>(S, P, rows, cols, sm_count, C, slice_cols, stream);
 }
 
+
+// ---- rows kept in REGISTERS across a cluster, the next row's slice already on its way --------------------------------
+// For rows beyond 32768 columns.  A CTA of NT threads holds a slice of up to 32 NT columns in registers (32 per thread,
+// as the register tier does for a whole row); its shared memory only receives the NEXT row's slice.  Each WARP owns a
+// contiguous piece of the slice (up to 4 KB): it waits for its piece alone, moves it to registers and at once issues
+// the bulk copy of the same piece of the next row, so no barrier sits in the load pipeline and the HBM read stream
+// does not pause for the reductions, the cluster exchange and the stores.  One read and one write per element, where
+// the two-read kernel moves every element through L2 twice.
+// CTAs of 512 threads, two per SM, whose phases overlap (CTAs of 1024 threads with slices of 32768 columns were slower
+// at every length: fewer clusters of them are resident at once, 15 of 8 CTAs against 14 of 16).
+constexpr int kRcThreads = 512;
+constexpr int kRcVecPerThread = 8;
+constexpr int kRcSliceMaxCols = kRcThreads * kRcVecPerThread * 4;                        // 16384
+constexpr long long kRcMaxCols = static_cast<long long>(kRcSliceMaxCols) * kMaxCluster;  // 262144
+constexpr uint32_t kSiteRcRowLoad = 121;
+constexpr uint32_t kSiteRcExchange = 122;
+
+struct RcControl {
+    uint64_t full[kRcThreads / 32];  // one per warp: its piece of the current row has landed
+    float red_max[kRcThreads / 32];
+    float red_sum[kRcThreads / 32];
+    uint64_t pairs_in[2];            // by row parity: the (maximum, sum) pairs of every CTA of the cluster have arrived
+    float2 xch[2][kMaxCluster];      // [row parity][CTA]: (local maximum, local sum)
+    uint32_t abort_flag;
+    uint32_t prior_failure;
+};
+constexpr int kRcControlBytes = 1024;
+static_assert(sizeof(RcControl) <= kRcControlBytes, "control block must fit its slot");
+
+template <typename OutT>
+__global__ void __launch_bounds__(kRcThreads, 2)
+softmax_rows_regcluster_kernel(const float* S, OutT* P, long long rows, long long cols, int slice_cols, int C) {
+    extern __shared__ __align__(16) uint8_t srs_smem[];
+    RcControl* ctl = reinterpret_cast<RcControl*>(srs_smem);
+    const float4* x = reinterpret_cast<const float4*>(srs_smem + kRcControlBytes);
+    volatile uint32_t* abort_flag = &ctl->abort_flag;
+
+    const uint32_t rank = C > 1 ? ptx::cluster_ctarank() : 0u;
+    const long long n_clusters = gridDim.x / C;
+    const long long cluster = blockIdx.x / C;
+    const long long c0 = static_cast<long long>(rank) * slice_cols;
+    const int n = static_cast<int>(c0 >= cols ? 0 : (cols - c0 < slice_cols ? cols - c0 : slice_cols));
+    const int nvec = n >> 2;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kWarpsRc = kRcThreads / 32;
+    const int piece = (nvec + kWarpsRc - 1) / kWarpsRc;  // vectors per warp, at most 256
+    const int v0 = warp * piece < nvec ? warp * piece : nvec;  // this warp's vectors: [v0, v1)
+    const int v1 = v0 + piece < nvec ? v0 + piece : nvec;
+    const uint32_t bytes = static_cast<uint32_t>(v1 - v0) * 16u;
+
+    if (threadIdx.x == 0) {
+        ctl->prior_failure = *reinterpret_cast<volatile unsigned int*>(&g_attnw_status);
+        for (int w = 0; w < kWarpsRc; ++w) ptx::mbar_init(&ctl->full[w], 1);
+        ptx::mbar_init(&ctl->pairs_in[0], 1);
+        ptx::mbar_init(&ctl->pairs_in[1], 1);
+        ctl->abort_flag = 0;
+        ptx::mbar_fence_init();
+    }
+    __syncthreads();
+    bool ok = ctl->prior_failure == 0u;
+    if (C > 1) {  // every CTA of the cluster runs before anyone writes into a peer
+        ptx::cluster_arrive_release();
+        ptx::cluster_wait_acquire();
+    }
+    auto issue = [&](long long row) {  // one lane: this warp's piece of `row` -> shared memory
+        ptx::mbar_expect_tx(&ctl->full[warp], bytes);
+        ptx::bulk_load_1d(ptx::smem_u32(x + v0), reinterpret_cast<const float4*>(S + row * cols + c0) + v0, bytes,
+                          &ctl->full[warp]);
+    };
+    if (ok && lane == 0 && bytes > 0 && cluster < rows) issue(cluster);
+
+    uint32_t it = 0;
+    for (long long row = cluster; row < rows; row += n_clusters, ++it) {
+        if (ok && bytes > 0) ok = fused_wait(&ctl->full[warp], it & 1u, abort_flag, kSiteRcRowLoad);
+        float4 v[kRcVecPerThread];
+        float m = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < kRcVecPerThread; ++k) {
+            const int idx = v0 + k * 32 + lane;
+            if (ok && idx < v1) {
+                v[k] = x[idx];
+                m = fmaxf(m, fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w)));
+            } else {
+                v[k] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            }
+        }
+        ptx::fence_proxy_async_smem();  // orders these reads before the next bulk copy into the same bytes
+        __syncwarp();
+        if (ok && lane == 0 && bytes > 0 && row + n_clusters < rows) issue(row + n_clusters);
+
+        m = sr_row_reduce<kRcThreads, true>(m, ctl->red_max);
+        // a warp that gave up has set the flag before the barrier inside the reduction: all or none of the CTA goes on
+        ok = *abort_flag == 0u && ctl->prior_failure == 0u;
+        const float mc = (m > -INFINITY) ? m : 0.0f;  // an empty slice (or a failure upstream): keeps inf - inf out
+        float l = 0.0f;
+#pragma unroll
+        for (int k = 0; k < kRcVecPerThread; ++k) {
+            // (x - m) first: the difference is exact near the maximum, so a constant row gives exactly 1
+            v[k].x = sr_ex2((v[k].x - mc) * kLog2e);
+            v[k].y = sr_ex2((v[k].y - mc) * kLog2e);
+            v[k].z = sr_ex2((v[k].z - mc) * kLog2e);
+            v[k].w = sr_ex2((v[k].w - mc) * kLog2e);
+            l += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+        }
+        l = sr_row_reduce<kRcThreads, false>(l, ctl->red_sum);
+
+        float factor;
+        if (C > 1) {
+            // One exchange of (maximum, sum) across the cluster without a cluster barrier: every CTA sends its pair into
+            // every CTA's slots (two sets by row parity) with a store that completes bytes on the receiver's mbarrier,
+            // and waits only for its own slots to fill.  A CTA can send the pair of row r + 2 (the same parity) only
+            // after receiving every pair of row r + 1, which its peers sent after reading their slots of row r.
+            const uint32_t par = it & 1u;
+            if (threadIdx.x < static_cast<unsigned>(C))
+                ptx::st_async_b64(ptx::map_to_cta(ptx::smem_u32(&ctl->xch[par][rank]), threadIdx.x), ptx::pack2(m, l),
+                                  ptx::map_to_cta(ptx::smem_u32(&ctl->pairs_in[par]), threadIdx.x));
+            if (threadIdx.x == 0) ptx::mbar_expect_tx(&ctl->pairs_in[par], static_cast<uint32_t>(C) * 8u);
+            if (ok) ok = fused_wait(&ctl->pairs_in[par], (it >> 1) & 1u, abort_flag, kSiteRcExchange);
+            float M = ctl->xch[par][0].x;
+            for (int c = 1; c < C; ++c) M = fmaxf(M, ctl->xch[par][c].x);
+            if (!(M > -INFINITY)) M = 0.0f;
+            float L = 0.0f;
+            for (int c = 0; c < C; ++c)  // the same order in every CTA; an empty slice has sum 0 and maximum -inf
+                L += ctl->xch[par][c].y * sr_ex2((ctl->xch[par][c].x - M) * kLog2e);
+            factor = sr_ex2((mc - M) * kLog2e) / L;
+        } else {
+            factor = 1.0f / l;
+        }
+        if (ok) {
+            OutT* dst = P + row * cols + c0;
+#pragma unroll
+            for (int k = 0; k < kRcVecPerThread; ++k) {
+                const int idx = v0 + k * 32 + lane;
+                if (idx < v1) sr_store4<OutT>(dst + 4ll * idx, v[k].x * factor, v[k].y * factor, v[k].z * factor, v[k].w * factor);
+            }
+        }
+    }
+    if (C > 1) {  // no CTA leaves while a peer may still write into its control block
+        ptx::cluster_arrive_release();
+        ptx::cluster_wait_acquire();
+    }
+}
+
+inline int rc_cluster_ctas_for(long long cols) {  // any size up to 16, not only powers of two
+    if (cols > kRcMaxCols) return 0;
+    return static_cast<int>((cols + kRcSliceMaxCols - 1) / kRcSliceMaxCols);
+}
+
+// `resident_clusters`: the caller's per-device memo of how many clusters of this size are resident at once (0 = not
+// asked yet, -1 = this cluster size cannot be launched here).
+template <typename OutT>
+inline cudaError_t launch_regcluster(const float* S, OutT* P, long long rows, long long cols, int* resident_clusters,
+                                     cudaStream_t stream) {
+    const int C = rc_cluster_ctas_for(cols);
+    if (C == 0) return cudaErrorInvalidValue;
+    constexpr int kSmemMax = kRcControlBytes + kRcSliceMaxCols * 4;
+    const int slice_cols = static_cast<int>(((cols / 4 + C - 1) / C) * 4);
+    auto kernel = softmax_rows_regcluster_kernel<OutT>;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kRcThreads);
+    cfg.dynamicSmemBytes = kRcControlBytes + static_cast<size_t>(slice_cols) * 4;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(C);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (*resident_clusters == 0) {  // once per device, output type and cluster size
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemMax);
+        if (e == cudaSuccess && C > 8) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        int n = 0;
+        if (e == cudaSuccess) {
+            cfg.gridDim = dim3(static_cast<unsigned>(C));
+            const size_t asked = cfg.dynamicSmemBytes;
+            cfg.dynamicSmemBytes = kSmemMax;  // the memo serves every row length of this cluster size
+            e = cudaOccupancyMaxActiveClusters(&n, kernel, &cfg);
+            cfg.dynamicSmemBytes = asked;
+        }
+        *resident_clusters = (e == cudaSuccess && n > 0) ? n : -1;
+        if (e != cudaSuccess) (void)cudaGetLastError();
+    }
+    if (*resident_clusters < 0) return cudaErrorInvalidConfiguration;
+    long long n_clusters = *resident_clusters;
+    if (n_clusters > rows) n_clusters = rows;
+    cfg.gridDim = dim3(static_cast<unsigned>(n_clusters * C));
+    return cudaLaunchKernelEx(&cfg, kernel, S, P, rows, cols, slice_cols, C);
+}
+
 }  // namespace srs
 }  // namespace attnw

@@ -20,9 +20,10 @@ def attnw():
 SHAPES = [(1, 4), (3, 8), (33, 36), (257, 100), (64, 128), (5, 132), (40, 260), (17, 1000), (9, 1024),
           (7, 1028), (6, 2052), (5, 4096), (4, 4100), (3, 8192), (3, 8196), (2, 16384), (2, 16388),
           (2, 32768), (3, 32772), (2, 70000), (600, 512),
-          # the shared-memory tier: one CTA, clusters of 2, 4, 8 and 16, more rows than clusters, its last column count;
-          # then the two-read tier beyond it
-          (5, 40000), (3, 49152), (2, 100000), (1, 196608), (300, 33000), (1, 393216), (2, 393220), (40, 98308)]
+          # beyond 32768 columns the rows live in the registers of a cluster of 3 to 16 CTAs (any size, ragged last slice,
+          # more rows than clusters, its last column count), then the two-read tier
+          (5, 40000), (3, 49152), (2, 100000), (1, 196608), (300, 33000), (1, 393216), (2, 393220), (40, 98308),
+          (9, 65536), (4, 81924), (150, 57348), (3, 180228), (3, 262144), (2, 262148), (33, 245764)]
 
 
 @pytest.mark.parametrize("rows,cols", SHAPES)
