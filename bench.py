@@ -305,6 +305,28 @@ def secondary_config(binding, inputs, name, peaks, steps=20, warmup=3):
     return out
 
 
+def long_rows_config(binding, peaks, steps=10, warmup=3):
+    """Row Softmax on long rows (the row-length axis of the paper's per-element runtime figure): 2^28 float32 scores
+    drawn on the device (values N(0, 3^2) as in c4; a timing-only line, parity is the tests' job) in rows of 32768 to
+    262144 columns; picoseconds per element against the copy roofline (6 bytes per element)."""
+    import torch
+    total = 1 << 28
+    g = torch.Generator(device="cuda")
+    g.manual_seed(4)
+    S = torch.empty(total, dtype=torch.float32, device="cuda")
+    S.normal_(0.0, 3.0, generator=g)
+    P = torch.empty(total, dtype=torch.bfloat16, device="cuda")
+    roof_ps = 6.0 / (peaks["hbm_gbs"] * 1e9) * 1e12
+    out = {"elements_per_launch": total, "roofline_ps_per_element": roof_ps, "steps": steps}
+    for cols in (32768, 65536, 131072, 262144):
+        s2, p2 = S.view(total // cols, cols), P.view(total // cols, cols)
+        ms = time_launches(lambda: binding.softmax_rows(s2, P=p2), steps, warmup, torch.cuda.synchronize) / steps
+        ps = ms * 1e-3 / total * 1e12
+        out[str(cols)] = {"ms": ms, "ps_per_element": ps, "roofline_frac": roof_ps / ps}
+    del S, P
+    return out
+
+
 def attention_config(binding, inputs, name, peaks, steps=20, warmup=3):
     """Short kernel-only measurement of attn_fused (the product with V, Section IV) on the shape of one of the
     configurations, with V drawn like K on its own stream (reported beside the headline, not part of it)."""
@@ -395,9 +417,10 @@ def run_profile_case(args):
         K = torch.empty_like(Q)
         fn = lambda: binding.project_qk(X, Wq, Wk, Q=Q, K=K)  # noqa: E731
         desc = f"attnw_project_qk B=1 N={w.N} d_model={dm} H={w.H} d={w.d}"
-    elif args.profile == "rows_long":
-        # rows beyond the register tier: kept in the shared memory of a cluster of two CTAs (32768 columns)
-        rows, cols = 4096, 32768
+    elif args.profile in ("rows_long", "rows_cluster"):
+        # rows beyond the register tier: kept in the shared memory of a cluster of two CTAs (32768 columns), or in the
+        # registers of a cluster of eight (131072 columns)
+        rows, cols = (4096, 32768) if args.profile == "rows_long" else (1024, 131072)
         w = inputs.Workload("rows-long", "rows", rows=rows, cols=cols, sigma=3.0, cfg_id=4)
         S = torch.from_numpy(inputs.make_scores(w, 0, rows)).cuda()
         P = torch.empty((rows, cols), dtype=torch.bfloat16, device="cuda")
@@ -601,6 +624,8 @@ def run_ours(args):
         for name in ("c4", "c5", "c2"):
             other[name] = secondary_config(binding, inputs, name, peaks)
             torch.cuda.empty_cache()
+        other["softmax_rows_long"] = long_rows_config(binding, peaks)
+        torch.cuda.empty_cache()
         other["attention_c3"] = attention_config(binding, inputs, "c3", peaks)
         torch.cuda.empty_cache()
         other["project_qk_c3"] = projection_config(binding, inputs, "c3", peaks)
@@ -628,7 +653,7 @@ def main():
     ap.add_argument("--sustained-seconds", type=float, default=2.0)
     ap.add_argument("--variant", choices=["auto", "two_pass", "resident", "gridrow"], default="auto",
                     help="kernel behind attnw_fused (see attnw_set_fused_variant)")
-    ap.add_argument("--profile", choices=["fused", "rows", "rows_long", "attention", "project"], default=None,
+    ap.add_argument("--profile", choices=["fused", "rows", "rows_long", "rows_cluster", "attention", "project"], default=None,
                     help="run a reduced case of one kernel for an ncu capture instead of the benchmark")
     ap.add_argument("--timeline", action="store_true",
                     help="per-phase cycle table of the headline kernel from an instrumented build (see timeline.py)")

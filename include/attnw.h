@@ -168,8 +168,8 @@ int softmax_rows_f32(const void* S, void* P, long long rows, long long cols, voi
  * Which form of the row Softmax softmax_rows uses (process-wide; Section VI-A compares the two on its hardware):
  *   0  by row length (default): rows of up to 262144 columns are read once and kept on chip ("caching": one
  *      exponential per element) - in registers up to 8192 columns, in the shared memory of one CTA up to 24576 and
- *      of a cluster of two CTAs up to 32768, in the registers of a cluster of 3 to 16 CTAs up to 262144; longer rows
- *      are read twice (the second time out of L2) and their exponentials recomputed
+ *      of a cluster of two CTAs up to 32768, in the registers of a cluster of 3 to 16 CTAs from 45057 to 262144;
+ *      rows in between and longer rows are read twice (the second time out of L2), their exponentials recomputed
  *   1  caching only: rows of up to 393216 columns are kept in the shared memory of a thread-block cluster of up to
  *      16 CTAs that exchange local maxima and sums through distributed shared memory; a call with cols > 393216
  *      returns ATTNW_ERR_UNSUPPORTED

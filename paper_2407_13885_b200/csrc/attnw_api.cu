@@ -692,8 +692,9 @@ int rows_entry(const void* S, void* P, long long rows, long long cols, void* str
         (void)cudaGetLastError();  // no cluster of that size on this device: fall through to the two-read kernel
         if (variant == 1) return ATTNW_ERR_UNSUPPORTED;
     }
-    // Rows of 32769 to 262144 columns: kept in the registers of a cluster, one read and one write per element.
-    if (variant == 0 && cols > kSoftmaxRowsRegTierMaxCols && cols <= srs::kRcMaxCols) {
+    // Rows of 45057 to 262144 columns: kept in the registers of a cluster, one read and one write per element
+    // (between 32769 and 45056 the slices of a cluster of three are short and the two-read kernel is ahead: measured).
+    if (variant == 0 && cols > kSoftmaxRowsRegClusterMinCols && cols <= srs::kRcMaxCols) {
         const int C = srs::rc_cluster_ctas_for(cols);
         const cudaError_t ce = srs::launch_regcluster<OutT>(static_cast<const float*>(S), static_cast<OutT*>(P), rows, cols,
                                                             &dev->rc_clusters[sizeof(OutT) == 4][C],

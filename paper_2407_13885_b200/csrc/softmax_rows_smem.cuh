@@ -16,6 +16,7 @@
 namespace attnw {
 
 constexpr long long kSoftmaxRowsSmemTierMinCols = 8192;  // rows longer than this may leave the register tier
+constexpr long long kSoftmaxRowsRegClusterMinCols = 45056;  // rows longer than this live in the registers of a cluster
 
 namespace srs {
 
@@ -256,6 +257,7 @@ softmax_rows_regcluster_kernel(const float* S, OutT* P, long long rows, long lon
     const int v0 = warp * piece < nvec ? warp * piece : nvec;  // this warp's vectors: [v0, v1)
     const int v1 = v0 + piece < nvec ? v0 + piece : nvec;
     const uint32_t bytes = static_cast<uint32_t>(v1 - v0) * 16u;
+    const bool full = v1 - v0 == kRcVecPerThread * 32;  // this warp's piece has all its 256 vectors
 
     if (threadIdx.x == 0) {
         ctl->prior_failure = *reinterpret_cast<volatile unsigned int*>(&g_attnw_status);
@@ -283,14 +285,22 @@ softmax_rows_regcluster_kernel(const float* S, OutT* P, long long rows, long lon
         if (ok && bytes > 0) ok = fused_wait(&ctl->full[warp], it & 1u, abort_flag, kSiteRcRowLoad);
         float4 v[kRcVecPerThread];
         float m = -INFINITY;
+        if (ok && full) {  // the common case, free of per-vector bounds checks
 #pragma unroll
-        for (int k = 0; k < kRcVecPerThread; ++k) {
-            const int idx = v0 + k * 32 + lane;
-            if (ok && idx < v1) {
-                v[k] = x[idx];
+            for (int k = 0; k < kRcVecPerThread; ++k) {
+                v[k] = x[v0 + k * 32 + lane];
                 m = fmaxf(m, fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w)));
-            } else {
-                v[k] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < kRcVecPerThread; ++k) {
+                const int idx = v0 + k * 32 + lane;
+                if (ok && idx < v1) {
+                    v[k] = x[idx];
+                    m = fmaxf(m, fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w)));
+                } else {
+                    v[k] = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+                }
             }
         }
         ptx::fence_proxy_async_smem();  // orders these reads before the next bulk copy into the same bytes
@@ -336,11 +346,16 @@ softmax_rows_regcluster_kernel(const float* S, OutT* P, long long rows, long lon
             factor = 1.0f / l;
         }
         if (ok) {
-            OutT* dst = P + row * cols + c0;
+            OutT* dst = P + row * cols + c0 + 4ll * (v0 + lane);
+            if (full) {
 #pragma unroll
-            for (int k = 0; k < kRcVecPerThread; ++k) {
-                const int idx = v0 + k * 32 + lane;
-                if (idx < v1) sr_store4<OutT>(dst + 4ll * idx, v[k].x * factor, v[k].y * factor, v[k].z * factor, v[k].w * factor);
+                for (int k = 0; k < kRcVecPerThread; ++k)
+                    sr_store4<OutT>(dst + 128 * k, v[k].x * factor, v[k].y * factor, v[k].z * factor, v[k].w * factor);
+            } else {
+#pragma unroll
+                for (int k = 0; k < kRcVecPerThread; ++k)
+                    if (v0 + k * 32 + lane < v1)
+                        sr_store4<OutT>(dst + 128 * k, v[k].x * factor, v[k].y * factor, v[k].z * factor, v[k].w * factor);
             }
         }
     }
