@@ -201,7 +201,8 @@ int attnw_host_release(void);
  * up records a code in a per-device status word, makes the kernel unwind and return normally, and the output of
  * that launch is then undefined.
  * The word is STICKY: while it is non-zero, every later launch of the tensor-core kernels (attnw_fused*, attn_fused,
- * attnw_project_qk) and of the shared-memory tier of softmax_rows* returns at once WITHOUT WRITING ITS OUTPUT - the
+ * attnw_project_qk) and of the shared-memory and cluster tiers of softmax_rows* (rows of 8193 to 32768 and of 45057
+ * to 262144 columns) returns at once WITHOUT WRITING ITS OUTPUT - the
  * call itself still returns ATTNW_OK, since it only enqueues - so that no work piles up behind a device that has
  * stopped making progress.  The register and streaming tiers of softmax_rows* have no waits and ignore the word.
  * attnw_query_status() synchronises `stream`, stores the word in *device_status (0 = no failure; otherwise
