@@ -43,6 +43,11 @@ def test_wait_runs_out_status_is_sticky_then_clears_and_work_resumes(attnw):
     attnw.softmax_rows(S, P=Pr)
     torch.cuda.synchronize()
     assert bool(torch.isnan(Pr).all())
+    Sc = torch.randn(8, 65536, device="cuda")          # ... and so does the cluster tier (registers of four CTAs)
+    Pc = torch.full((8, 65536), float("nan"), dtype=torch.bfloat16, device="cuda")
+    attnw.softmax_rows(Sc, P=Pc)
+    torch.cuda.synchronize()
+    assert bool(torch.isnan(Pc).all())
 
     # the query reports the failure with the site of the wait, once
     word = attnw.query_status()
@@ -59,6 +64,9 @@ def test_wait_runs_out_status_is_sticky_then_clears_and_work_resumes(attnw):
             attnw.set_fused_variant("auto")
         torch.cuda.synchronize()
         assert_close_to_oracle(P, ref, f"{variant} after the status was cleared")
+    attnw.softmax_rows(Sc, P=Pc)
+    torch.cuda.synchronize()
+    assert_close_to_oracle(Pc, oracle.softmax_rows(Sc.cpu().numpy()), "cluster tier after the status was cleared")
     assert attnw.query_status() == 0
 
 
